@@ -1,0 +1,127 @@
+/*
+ * s2a -- shifted sparse attention (S2-Attn) for NVIDIA B200 (sm_100a), forward and backward.
+ *
+ * The operation is the one LongLoRA states in Algorithm 1 and Section 3.2, with the attention of
+ * Eq. 1 inside each group:
+ *   - the N tokens of a sequence are cut into N/G groups of G consecutive tokens;
+ *   - in the second half of the heads (h >= H/2) the tokens are rolled by -G/2 first, so that the
+ *     group boundaries sit half a group later and the last group wraps around the sequence end
+ *     (Algorithm 1, key line 1; Section 3.2: with N=8192, G=2048 the first shifted group holds
+ *     tokens 1025..3072 and the first and last 1024 tokens share a group);
+ *   - causal softmax attention, scores scaled by 1/sqrt(d), runs inside each group in rolled order;
+ *   - the second half of the heads is rolled back by +G/2 (key line 2), so every output is indexed
+ *     by ORIGINAL token position.
+ * Grouped-query attention: query head h reads KV head floor(h / (H/Hkv)) at the same (rolled)
+ * coordinates as itself.  The wrapped group of a shifted head is kept as the paper's default
+ * method has it: its first-half tokens attend the sequence's last G/2 tokens.
+ *
+ * Conventions shared by all entry points
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller unless a function says "host".
+ *     The library never allocates, frees or keeps them.  All tensors are dense, last index fastest.
+ *   - q, o, dO, dq : bf16 [B, N, H,   d]
+ *     k, v, dk, dv : bf16 [B, N, Hkv, d]
+ *     lse          : fp32 [B, H, N]   natural-log sum-exp of the scaled scores, original token order
+ *   - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).  Calls only enqueue
+ *     work and return without synchronising.
+ *   - Return value: S2A_OK (0) or a negative s2a_status.  On error nothing was enqueued.
+ *   - Supported shapes: d in {64, 128}; G a multiple of 256 (so that G/2 is a whole number of
+ *     128-token tiles); N a multiple of G; H even; H a multiple of Hkv; pointers 16-byte aligned;
+ *     a device of compute capability 10.x.  Anything else is rejected, never approximated.
+ *   - Device-side waits are bounded.  If one ever expires the kernel records where, stops cleanly,
+ *     and s2a_device_status() reports it; outputs of that launch are then undefined.
+ */
+#ifndef S2A_H_
+#define S2A_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum s2a_status {
+    S2A_OK = 0,
+    S2A_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, N % G, odd G or H, H % Hkv, misaligned pointer, small workspace */
+    S2A_ERR_UNSUPPORTED = -2, /* d not in {64,128}, G not a multiple of 256, device is not sm_100 */
+    S2A_ERR_CUDA = -3,        /* a CUDA call failed while enqueuing; see s2a_last_cuda_error() */
+    S2A_ERR_TIMEOUT = -4      /* reported by s2a_device_status(): a bounded device-side wait expired */
+} s2a_status;
+
+/*
+ * Forward (Algorithm 1 with Eq. 1 inside each group).
+ *   in : q, k, v                     out: o (bf16, rounded once from fp32), lse (fp32)
+ * Scores and the P.V product accumulate in fp32 on the tensor cores; P is rounded to bf16 before
+ * the second product.  One kernel launch on `stream`.
+ */
+int s2a_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
+            int B, int N, int H, int Hkv, int d, int G, void* stream);
+
+/*
+ * Backward: gradients of sum(o * dO) with respect to q, k, v (the paper trains through
+ * Algorithm 1 by automatic differentiation; this is that derivative written out).
+ *   in : q, k, v, o, lse (o and lse exactly as s2a_fwd produced them), dO
+ *   out: dq, dk, dv (overwritten, not accumulated into)
+ *   workspace: caller-owned device scratch of at least s2a_bwd_workspace_bytes(...) bytes,
+ *              256-byte aligned; holds D[b,h,t] = dO[b,t,h,:] . o[b,t,h,:] in fp32.
+ * dk and dv sum over the H/Hkv query heads that share a KV head inside one thread block, so the
+ * result is deterministic (no atomics).  Three kernel launches on `stream`.
+ */
+int s2a_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO,
+            void* dq, void* dk, void* dv,
+            int B, int N, int H, int Hkv, int d, int G,
+            void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of scratch s2a_bwd needs for these sizes (0 if the sizes are invalid). */
+size_t s2a_bwd_workspace_bytes(int B, int N, int H, int Hkv, int d, int G);
+
+/*
+ * Generalised forms (Section 3.2 pilot study, Table 6 and Appendix B variant 1): the first
+ * `n_unshifted` heads use the unshifted partition, the remaining heads are rolled by -shift
+ * tokens (shift a multiple of 128, |shift| < N; the paper's method is n_unshifted = H/2,
+ * shift = G/2).  n_unshifted = H gives "pattern 1 only"; with G = N as well it is ordinary full
+ * causal attention, which the fine-tuned model uses at inference.  `scale` multiplies the scores
+ * (pass 1/sqrt(d) for the standard choice).  H may be odd here.
+ */
+int s2a_fwd_ex(const void* q, const void* k, const void* v, void* o, float* lse,
+               int B, int N, int H, int Hkv, int d, int G,
+               float scale, int n_unshifted, int shift, void* stream);
+int s2a_bwd_ex(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO,
+               void* dq, void* dk, void* dv,
+               int B, int N, int H, int Hkv, int d, int G,
+               float scale, int n_unshifted, int shift,
+               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Forward + backward from HOST buffers (pinned memory recommended): copies q, k, v, dO to the
+ * caller's device buffers, runs s2a_fwd and s2a_bwd, and copies o, lse, dq, dk, dv back, all
+ * enqueued on `stream`; the caller synchronises the stream before reading the host outputs.
+ *   h_*  : host pointers, same layouts and types as the device tensors
+ *   d_*  : device buffers of the same sizes, owned by the caller (the library allocates nothing)
+ */
+int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const void* h_dO,
+                     void* h_o, float* h_lse, void* h_dq, void* h_dk, void* h_dv,
+                     void* d_q, void* d_k, void* d_v, void* d_dO, void* d_o, float* d_lse,
+                     void* d_dq, void* d_dk, void* d_dv,
+                     int B, int N, int H, int Hkv, int d, int G,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Reads (and clears) the device-side status word of the current device.  Synchronises the device.
+ * Returns S2A_OK, S2A_ERR_TIMEOUT (a bounded wait expired in some kernel since the last call; if
+ * `where` is non-NULL it receives a code naming the kernel and the wait), or S2A_ERR_CUDA.
+ */
+int s2a_device_status(int* where);
+
+/* Static, human-readable text for a status code. */
+const char* s2a_status_string(int status);
+
+/* cudaError_t value of the most recent failing CUDA call made by this library on this thread. */
+int s2a_last_cuda_error(void);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int s2a_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* S2A_H_ */

@@ -1,0 +1,289 @@
+// Host side of the C-ABI declared in include/s2a.h: argument validation, TMA tensor maps,
+// kernel launches.  Nothing here allocates device memory.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include "../../include/s2a.h"
+#include "s2a_params.h"
+
+namespace s2a {
+namespace {
+
+// Device-wide status word written by kernels whose bounded wait expired (one copy per device
+// that loads this library).
+__device__ int g_status_word;
+
+thread_local int tl_last_cuda_error = 0;
+
+constexpr int kMaxDevices = 64;
+struct DeviceState {
+    bool ready = false;
+    int* status_ptr = nullptr;
+};
+DeviceState g_dev[kMaxDevices];
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+int cuda_fail(cudaError_t e) {
+    tl_last_cuda_error = static_cast<int>(e);
+    return S2A_ERR_CUDA;
+}
+
+// Per-device set-up: architecture check, shared-memory attributes, address of the status word.
+int prepare_device(DeviceState** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return S2A_ERR_UNSUPPORTED;
+    DeviceState& ds = g_dev[dev];
+    if (!ds.ready) {
+        int major = 0;
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (major != 10) return S2A_ERR_UNSUPPORTED;
+        if (!g_encode) {
+            void* fn = nullptr;
+            cudaDriverEntryPointQueryResult qres;
+            e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+            if (e != cudaSuccess) return cuda_fail(e);
+            if (qres != cudaDriverEntryPointSuccess || !fn) return cuda_fail(cudaErrorNotSupported);
+            g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+        }
+        e = configure_fwd();
+        if (e != cudaSuccess) return cuda_fail(e);
+        e = configure_bwd();
+        if (e != cudaSuccess) return cuda_fail(e);
+        e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ds.status_ptr), g_status_word);
+        if (e != cudaSuccess) return cuda_fail(e);
+        ds.ready = true;
+    }
+    *out = &ds;
+    return S2A_OK;
+}
+
+// bf16 tensor [B, N, heads, d] viewed as (d, heads, N, B); box = 64 columns x `box_rows` tokens of
+// one head, written to shared memory with the 128-byte swizzle the MMA descriptors expect.
+int make_tmap(CUtensorMap* tm, const void* base, int d, int heads, int N, int B, int box_rows) {
+    const cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)heads, (cuuint64_t)N, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)d * 2, (cuuint64_t)heads * d * 2, (cuuint64_t)N * heads * d * 2};
+    const cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        tl_last_cuda_error = static_cast<int>(cudaErrorInvalidValue);
+        return S2A_ERR_CUDA;
+    }
+    return S2A_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(int B, int N, int H, int Hkv, int d, int G, float scale, int n_unshifted, int shift) {
+    if (B <= 0 || N <= 0 || H <= 0 || Hkv <= 0 || d <= 0 || G <= 0) return S2A_ERR_INVALID_ARG;
+    if (N % G != 0 || H % Hkv != 0) return S2A_ERR_INVALID_ARG;
+    if (n_unshifted < 0 || n_unshifted > H) return S2A_ERR_INVALID_ARG;
+    if (!(scale > 0.f) || !isfinite(scale)) return S2A_ERR_INVALID_ARG;
+    if (shift <= -N || shift >= N) return S2A_ERR_INVALID_ARG;
+    if (d != 64 && d != 128) return S2A_ERR_UNSUPPORTED;
+    if (G % kTile != 0 || shift % kTile != 0) return S2A_ERR_UNSUPPORTED;
+    // grid sizes and 32-bit token arithmetic
+    const long long tiles = (long long)B * H * (N / kTile);
+    if (tiles > 0x7fffffffLL || (long long)N + G >= 0x40000000LL) return S2A_ERR_UNSUPPORTED;
+    return S2A_OK;
+}
+
+Geometry make_geometry(int B, int N, int H, int Hkv, int G, int n_unshifted, int shift) {
+    Geometry g;
+    g.B = B, g.N = N, g.H = H, g.Hkv = Hkv, g.G = G;
+    g.n_unshifted = n_unshifted;
+    g.shift = shift;
+    g.tiles_per_group = G / kTile;
+    g.groups = N / G;
+    return g;
+}
+
+constexpr float kLog2eHost = 1.4426950408889634f;
+
+}  // namespace
+}  // namespace s2a
+
+using namespace s2a;
+
+#pragma GCC visibility push(default)
+extern "C" {
+
+int s2a_version(void) { return 100; }
+
+int s2a_last_cuda_error(void) { return tl_last_cuda_error; }
+
+const char* s2a_status_string(int status) {
+    switch (status) {
+        case S2A_OK: return "ok";
+        case S2A_ERR_INVALID_ARG: return "invalid argument (null or misaligned pointer, bad size, or workspace too small)";
+        case S2A_ERR_UNSUPPORTED: return "unsupported shape or device (need d in {64,128}, G and shift multiples of 128, sm_100)";
+        case S2A_ERR_CUDA: return "a CUDA call failed; see s2a_last_cuda_error()";
+        case S2A_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+int s2a_fwd_ex(const void* q, const void* k, const void* v, void* o, float* lse, int B, int N, int H, int Hkv, int d,
+               int G, float scale, int n_unshifted, int shift, void* stream) {
+    if (!q || !k || !v || !o || !lse) return S2A_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return S2A_ERR_INVALID_ARG;
+    int rc = check_shape(B, N, H, Hkv, d, G, scale, n_unshifted, shift);
+    if (rc != S2A_OK) return rc;
+    DeviceState* ds = nullptr;
+    rc = prepare_device(&ds);
+    if (rc != S2A_OK) return rc;
+
+    FwdParams p;
+    memset(&p, 0, sizeof p);
+    if ((rc = make_tmap(&p.tm_q, q, d, H, N, B, kTile)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&p.tm_k, k, d, Hkv, N, B, kTile)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&p.tm_v, v, d, Hkv, N, B, kTile)) != S2A_OK) return rc;
+    p.o = static_cast<__nv_bfloat16*>(o);
+    p.lse = lse;
+    p.status = ds->status_ptr;
+    p.geo = make_geometry(B, N, H, Hkv, G, n_unshifted, shift);
+    p.scale_log2 = scale * kLog2eHost;
+    cudaError_t e = launch_fwd(p, d, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? S2A_OK : cuda_fail(e);
+}
+
+int s2a_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int N, int H, int Hkv, int d,
+            int G, void* stream) {
+    if (d <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
+    if (G % (2 * kTile) != 0) return (G > 0 && N > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
+    return s2a_fwd_ex(q, k, v, o, lse, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2, G / 2, stream);
+}
+
+size_t s2a_bwd_workspace_bytes(int B, int N, int H, int Hkv, int d, int G) {
+    if (B <= 0 || N <= 0 || H <= 0 || Hkv <= 0 || d <= 0 || G <= 0) return 0;
+    if (N % G != 0 || H % Hkv != 0) return 0;
+    const size_t bytes = static_cast<size_t>(B) * H * N * sizeof(float);
+    return (bytes + 255) & ~static_cast<size_t>(255);
+}
+
+int s2a_bwd_ex(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO, void* dq,
+               void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, float scale, int n_unshifted,
+               int shift, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!q || !k || !v || !o || !lse || !dO || !dq || !dk || !dv || !workspace) return S2A_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse) || !aligned16(dO) ||
+        !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
+        return S2A_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return S2A_ERR_INVALID_ARG;
+    int rc = check_shape(B, N, H, Hkv, d, G, scale, n_unshifted, shift);
+    if (rc != S2A_OK) return rc;
+    if (workspace_bytes < s2a_bwd_workspace_bytes(B, N, H, Hkv, d, G)) return S2A_ERR_INVALID_ARG;
+    DeviceState* ds = nullptr;
+    rc = prepare_device(&ds);
+    if (rc != S2A_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const Geometry geo = make_geometry(B, N, H, Hkv, G, n_unshifted, shift);
+    float* Dsum = static_cast<float*>(workspace);
+
+    BwdDqParams pq;
+    memset(&pq, 0, sizeof pq);
+    if ((rc = make_tmap(&pq.tm_q, q, d, H, N, B, kTile)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pq.tm_do, dO, d, H, N, B, kTile)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pq.tm_k, k, d, Hkv, N, B, kSubTile)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pq.tm_v, v, d, Hkv, N, B, kSubTile)) != S2A_OK) return rc;
+    pq.lse = lse, pq.Dsum = Dsum, pq.dq = static_cast<__nv_bfloat16*>(dq);
+    pq.status = ds->status_ptr, pq.geo = geo, pq.scale = scale, pq.scale_log2 = scale * kLog2eHost;
+
+    BwdDkDvParams pk;
+    memset(&pk, 0, sizeof pk);
+    if ((rc = make_tmap(&pk.tm_k, k, d, Hkv, N, B, kTile)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pk.tm_v, v, d, Hkv, N, B, kTile)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pk.tm_q, q, d, H, N, B, kSubTile)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pk.tm_do, dO, d, H, N, B, kSubTile)) != S2A_OK) return rc;
+    pk.lse = lse, pk.Dsum = Dsum;
+    pk.dk = static_cast<__nv_bfloat16*>(dk), pk.dv = static_cast<__nv_bfloat16*>(dv);
+    pk.status = ds->status_ptr, pk.geo = geo, pk.scale = scale, pk.scale_log2 = scale * kLog2eHost;
+
+    PreParams pp;
+    pp.o = static_cast<const __nv_bfloat16*>(o), pp.dO = static_cast<const __nv_bfloat16*>(dO), pp.Dsum = Dsum;
+    pp.B = B, pp.N = N, pp.H = H;
+
+    cudaError_t e = launch_bwd_preprocess(pp, d, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = launch_bwd_dkdv(pk, d, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = launch_bwd_dq(pq, d, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return S2A_OK;
+}
+
+int s2a_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO, void* dq,
+            void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, void* workspace, size_t workspace_bytes,
+            void* stream) {
+    if (d <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
+    if (G % (2 * kTile) != 0) return (G > 0 && N > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
+    return s2a_bwd_ex(q, k, v, o, lse, dO, dq, dk, dv, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2,
+                      G / 2, workspace, workspace_bytes, stream);
+}
+
+int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const void* h_dO, void* h_o, float* h_lse,
+                     void* h_dq, void* h_dk, void* h_dv, void* d_q, void* d_k, void* d_v, void* d_dO, void* d_o,
+                     float* d_lse, void* d_dq, void* d_dk, void* d_dv, int B, int N, int H, int Hkv, int d, int G,
+                     void* workspace, size_t workspace_bytes, void* stream) {
+    if (!h_q || !h_k || !h_v || !h_dO || !h_o || !h_lse || !h_dq || !h_dk || !h_dv) return S2A_ERR_INVALID_ARG;
+    if (!d_q || !d_k || !d_v || !d_dO || !d_o || !d_lse || !d_dq || !d_dk || !d_dv) return S2A_ERR_INVALID_ARG;
+    if (d <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
+    int rc = check_shape(B, N, H, Hkv, d, G, 1.0f, H / 2, G / 2);
+    if (rc != S2A_OK) return rc;
+    if (G % (2 * kTile) != 0) return S2A_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < s2a_bwd_workspace_bytes(B, N, H, Hkv, d, G)) return S2A_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t nq = static_cast<size_t>(B) * N * H * d * 2;
+    const size_t nk = static_cast<size_t>(B) * N * Hkv * d * 2;
+    const size_t nl = static_cast<size_t>(B) * H * N * sizeof(float);
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(d_q, h_q, nq, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(d_k, h_k, nk, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(d_v, h_v, nk, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(d_dO, h_dO, nq, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+    rc = s2a_fwd(d_q, d_k, d_v, d_o, d_lse, B, N, H, Hkv, d, G, stream);
+    if (rc != S2A_OK) return rc;
+    rc = s2a_bwd(d_q, d_k, d_v, d_o, d_lse, d_dO, d_dq, d_dk, d_dv, B, N, H, Hkv, d, G, workspace, workspace_bytes,
+                 stream);
+    if (rc != S2A_OK) return rc;
+    if ((e = cudaMemcpyAsync(h_o, d_o, nq, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(h_lse, d_lse, nl, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(h_dq, d_dq, nq, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(h_dk, d_dk, nk, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(h_dv, d_dv, nk, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+    return S2A_OK;
+}
+
+int s2a_device_status(int* where) {
+    DeviceState* ds = nullptr;
+    int rc = prepare_device(&ds);
+    if (rc != S2A_OK) return rc;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e);
+    int word = 0;
+    e = cudaMemcpy(&word, ds->status_ptr, sizeof word, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (word != 0) {
+        const int zero = 0;
+        e = cudaMemcpy(ds->status_ptr, &zero, sizeof zero, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (where) *where = word;
+        return S2A_ERR_TIMEOUT;
+    }
+    if (where) *where = 0;
+    return S2A_OK;
+}
+
+}  // extern "C"
+#pragma GCC visibility pop

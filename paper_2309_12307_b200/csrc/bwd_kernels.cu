@@ -1,0 +1,612 @@
+// S2-Attn backward for sm_100a: the derivative of Algorithm 1 (with Eq. 1 inside each group).
+//
+// With P = exp(scale * Q K^T - lse) on the attended pairs and D_t = dO_t . o_t:
+//     dV = P^T dO          dP = dO V^T          dS = P o (dP - D)
+//     dQ = scale * dS K    dK = scale * dS^T Q
+// Three kernels:
+//   1. preprocess: D[b,h,t] = sum_c dO[b,t,h,c] * o[b,t,h,c]                     (memory bound)
+//   2. dQ:   one CTA per 128-row query tile, streams 64-key sub-tiles of its group (keys <= query)
+//   3. dK,dV: one CTA per 128-row key tile, streams 64-query sub-tiles of every query head that
+//            shares the KV head (queries >= key), so the sum over those heads stays in tensor
+//            memory and needs no atomics.  It works on the transposed scores S^T = K Q^T so that
+//            P^T and dS^T come out with keys along tensor-memory lanes, which is the layout the
+//            A operand of dV += P^T dO and dK += dS^T Q needs.
+// The roll of the shifted heads and the group boundaries are folded into TMA coordinates exactly
+// as in the forward kernel; all results are stored at original token rows.
+//
+// Both tensor-core kernels share one software pipeline (192 threads, one CTA per SM): warp 0
+// loads with TMA, warp 1 issues tcgen05 MMAs, warps 2-5 do the elementwise work with one
+// tensor-memory lane per thread.  The two score products of step n+1 are issued before the
+// gradient products of step n, into the other half of a double buffer, so the elementwise work
+// of step n overlaps tensor-core work.
+#include "s2a_params.h"
+#include "sm100_ptx.cuh"
+
+namespace s2a {
+
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+__device__ __forceinline__ int mod_pos(int x, int n) {
+    int r = x % n;
+    return r < 0 ? r + n : r;
+}
+
+// ------------------------------------------------------------------------------------------------
+// 1. preprocess
+// ------------------------------------------------------------------------------------------------
+// Each row of d bf16 values is read by d/8 threads with 16-byte loads.
+template <int HD>
+__global__ void __launch_bounds__(256) s2a_bwd_preprocess_kernel(const PreParams p) {
+    constexpr int kThreadsPerRow = HD / 8;
+    const long long n_rows = static_cast<long long>(p.B) * p.N * p.H;
+    const long long gtid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const long long row = gtid / kThreadsPerRow;  // (b * N + t) * H + h
+    const int part = static_cast<int>(gtid % kThreadsPerRow);
+    float acc = 0.f;
+    if (row < n_rows) {
+        const uint4 a = reinterpret_cast<const uint4*>(p.o + row * HD)[part];
+        const uint4 c = reinterpret_cast<const uint4*>(p.dO + row * HD)[part];
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
+        const uint32_t cw[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            // a bf16 is the upper half of an fp32
+            acc = fmaf(__uint_as_float(aw[e] << 16), __uint_as_float(cw[e] << 16), acc);
+            acc = fmaf(__uint_as_float(aw[e] & 0xffff0000u), __uint_as_float(cw[e] & 0xffff0000u), acc);
+        }
+    }
+#pragma unroll
+    for (int off = kThreadsPerRow / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (row < n_rows && part == 0) {
+        const int h = static_cast<int>(row % p.H);
+        const long long bt = row / p.H;
+        const int t = static_cast<int>(bt % p.N);
+        const long long b = bt / p.N;
+        p.Dsum[(b * p.H + h) * p.N + t] = acc;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// shared configuration of the two tensor-core kernels
+// ------------------------------------------------------------------------------------------------
+template <int HD>
+struct BwdCfg {
+    static constexpr int kThreads = 192;
+    static constexpr int kBoxes = HD / 64;
+    static constexpr int kBigBoxBytes = kTile * 128;            // 128-row box
+    static constexpr int kSubBoxBytes = kSubTile * 128;         // 64-row box
+    static constexpr int kBigTileBytes = kBoxes * kBigBoxBytes; // resident operand tile
+    static constexpr int kSubTileBytes = kBoxes * kSubBoxBytes; // streamed operand tile
+    static constexpr int kStages = 4;
+    static constexpr int kStatBytes = kSubTile * 4;             // lse or D of one streamed tile
+    static constexpr int kStageBytes = 2 * kSubTileBytes;       // two streamed operands per stage
+    static constexpr int kBarBytes = 512;
+    static constexpr int kNeeded = 1024 + 2 * kBigTileBytes + kStages * kStageBytes + kStages * 2 * kStatBytes + kBarBytes;
+    // at least 120 KB so that only one CTA fits on an SM: each CTA allocates all of tensor memory
+    static constexpr int kSmemBytes = kNeeded > 120 * 1024 ? kNeeded : 120 * 1024;
+    static constexpr int kTmemCols = 512;
+};
+
+// Pack 32 fp32 values (as raw bits) into 16 bf16x2 words.
+__device__ __forceinline__ void pack32(const float (&x)[32], uint32_t (&out)[16]) {
+#pragma unroll
+    for (int e = 0; e < 16; ++e) out[e] = pack_bf16(x[2 * e], x[2 * e + 1]);
+}
+
+// Store one accumulator row (HD fp32 columns in tensor memory, times `mul`) as bf16.
+template <int HD>
+__device__ __forceinline__ void store_acc_row(uint32_t t_addr, float mul, __nv_bfloat16* dst_row) {
+#pragma unroll
+    for (int c = 0; c < HD / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32(t_addr + c * 32, r);
+        tmem_wait_ld();
+        uint4* dst = reinterpret_cast<uint4*>(dst_row + c * 32);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            uint4 pk;
+            pk.x = pack_bf16(__uint_as_float(r[8 * e + 0]) * mul, __uint_as_float(r[8 * e + 1]) * mul);
+            pk.y = pack_bf16(__uint_as_float(r[8 * e + 2]) * mul, __uint_as_float(r[8 * e + 3]) * mul);
+            pk.z = pack_bf16(__uint_as_float(r[8 * e + 4]) * mul, __uint_as_float(r[8 * e + 5]) * mul);
+            pk.w = pack_bf16(__uint_as_float(r[8 * e + 6]) * mul, __uint_as_float(r[8 * e + 7]) * mul);
+            dst[e] = pk;
+        }
+    }
+}
+
+// Barrier block common to both kernels.
+template <int kStages>
+struct BwdBars {
+    uint64_t res_full;            // resident operands landed
+    uint64_t acc_full;            // all gradient MMAs done
+    uint64_t drain;               // abort path only
+    uint64_t s_full[2];           // score products of a step are in tensor memory
+    uint64_t p_full[2];           // bf16 P / dS of a step are in tensor memory
+    uint64_t st_full[kStages];    // streamed operands of a stage landed
+    uint64_t st_empty[kStages];   // MMAs reading a stage are done
+    uint32_t tmem_slot;
+    int abort_flag;
+};
+
+// ------------------------------------------------------------------------------------------------
+// 2. dQ
+// ------------------------------------------------------------------------------------------------
+// Tensor memory columns: dQ [0,HD)   S buffers [128,192) [192,256)   dP buffers [256,320) [320,384)
+template <int HD>
+__global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(const __grid_constant__ BwdDqParams p) {
+    using C = BwdCfg<HD>;
+    using Bars = BwdBars<C::kStages>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sQ = smem;                                // resident: Q_i
+    uint8_t* sDO = sQ + C::kBigTileBytes;              // resident: dO_i
+    uint8_t* sStage = sDO + C::kBigTileBytes;          // per stage: K_n then V_n
+    Bars* bars = reinterpret_cast<Bars*>(sStage + C::kStages * C::kStageBytes + C::kStages * 2 * C::kStatBytes);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const Geometry& geo = p.geo;
+
+    const int Tg = geo.tiles_per_group;
+    const int i = Tg - 1 - static_cast<int>(blockIdx.x % Tg);  // heaviest query tiles first
+    const int unit = blockIdx.x / Tg;
+    const int g = unit % geo.groups;
+    const int h = (unit / geo.groups) % geo.H;
+    const int b = unit / (geo.groups * geo.H);
+    const int hk = h / (geo.H / geo.Hkv);
+    const int s = (h < geo.n_unshifted) ? 0 : geo.shift;
+    const int n_steps = 2 * (i + 1);  // key sub-tiles 0 .. 2i+1 of the group
+    const int tq0 = mod_pos(g * geo.G + i * kTile + s, geo.N);
+
+    if (threadIdx.x == 0) {
+        mbar_init(&bars->res_full, 1);
+        mbar_init(&bars->acc_full, 1);
+        mbar_init(&bars->drain, 1);
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(&bars->s_full[x], 1);
+            mbar_init(&bars->p_full[x], 128);
+        }
+        for (int st = 0; st < C::kStages; ++st) {
+            mbar_init(&bars->st_full[st], 1);
+            mbar_init(&bars->st_empty[st], 1);
+        }
+        bars->abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&p.tm_q);
+        tma_prefetch_desc(&p.tm_do);
+        tma_prefetch_desc(&p.tm_k);
+        tma_prefetch_desc(&p.tm_v);
+    }
+    if (warp == 1) {
+        tmem_alloc(&bars->tmem_slot, C::kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = bars->tmem_slot;
+    const WaitCtx ctx{&bars->abort_flag, p.status};
+    constexpr uint32_t kColAcc = 0, kColS = 128, kColP = 256;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_expect_tx(&bars->res_full, 2 * C::kBigTileBytes);
+            for (int bx = 0; bx < C::kBoxes; ++bx) {
+                tma_load_4d(sQ + bx * C::kBigBoxBytes, &p.tm_q, &bars->res_full, bx * 64, h, tq0, b);
+                tma_load_4d(sDO + bx * C::kBigBoxBytes, &p.tm_do, &bars->res_full, bx * 64, h, tq0, b);
+            }
+            int n = 0;
+            for (; n < n_steps; ++n) {
+                const int st = n % C::kStages;
+                const uint32_t ph = (n / C::kStages) & 1;
+                const int tk0 = mod_pos(g * geo.G + n * kSubTile + s, geo.N);
+                if (!mbar_wait(&bars->st_empty[st], ph ^ 1, ctx, kWaitBwdDq + 1)) break;
+                mbar_expect_tx(&bars->st_full[st], C::kStageBytes);
+                uint8_t* sK = sStage + st * C::kStageBytes;
+                uint8_t* sV = sK + C::kSubTileBytes;
+                for (int bx = 0; bx < C::kBoxes; ++bx) {
+                    tma_load_4d(sK + bx * C::kSubBoxBytes, &p.tm_k, &bars->st_full[st], bx * 64, hk, tk0, b);
+                    tma_load_4d(sV + bx * C::kSubBoxBytes, &p.tm_v, &bars->st_full[st], bx * 64, hk, tk0, b);
+                }
+            }
+            if (bars->abort_flag != 0) {
+                mbar_wait_drain(&bars->res_full, 0);
+                for (int nn = (n > C::kStages ? n - C::kStages : 0); nn < n; ++nn)
+                    mbar_wait_drain(&bars->st_full[nn % C::kStages], (nn / C::kStages) & 1);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);  // S = Q K^T, dP = dO V^T
+            constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);       // dQ += dS K   (K is MN-major)
+            const uint32_t aQ = smem_u32(sQ), aDO = smem_u32(sDO);
+            // score products of step n into buffer n & 1
+            auto issue_scores = [&](int n) -> bool {
+                const int st = n % C::kStages;
+                if (!mbar_wait(&bars->st_full[st], (n / C::kStages) & 1, ctx, kWaitBwdDq + 2)) return false;
+                tc_fence_after();
+                const uint32_t aK = smem_u32(sStage + st * C::kStageBytes);
+                const uint32_t aV = aK + C::kSubTileBytes;
+                const uint32_t tS = tmem_base + kColS + (n & 1) * kSubTile;
+                const uint32_t tP = tmem_base + kColP + (n & 1) * kSubTile;
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t offA = (kk >> 2) * C::kBigBoxBytes + (kk & 3) * 32;
+                    const uint32_t offB = (kk >> 2) * C::kSubBoxBytes + (kk & 3) * 32;
+                    mma_ss(tS, desc_k_major(aQ + offA), desc_k_major(aK + offB), idesc_sc, kk > 0);
+                }
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t offA = (kk >> 2) * C::kBigBoxBytes + (kk & 3) * 32;
+                    const uint32_t offB = (kk >> 2) * C::kSubBoxBytes + (kk & 3) * 32;
+                    mma_ss(tP, desc_k_major(aDO + offA), desc_k_major(aV + offB), idesc_sc, kk > 0);
+                }
+                mma_commit(&bars->s_full[n & 1]);
+                return true;
+            };
+            bool ok = mbar_wait(&bars->res_full, 0, ctx, kWaitBwdDq + 3);
+            ok = ok && issue_scores(0);
+            for (int n = 0; ok && n < n_steps; ++n) {
+                if (n + 1 < n_steps && !issue_scores(n + 1)) break;
+                if (!mbar_wait(&bars->p_full[n & 1], (n >> 1) & 1, ctx, kWaitBwdDq + 4)) break;
+                tc_fence_after();
+                const int st = n % C::kStages;
+                const uint32_t aK = smem_u32(sStage + st * C::kStageBytes);
+                const uint32_t tdS = tmem_base + kColS + (n & 1) * kSubTile;  // bf16 dS over the S buffer
+#pragma unroll
+                for (int kk = 0; kk < kSubTile / 16; ++kk)
+                    mma_ts(tmem_base + kColAcc, tdS + kk * 8, desc_mn_major(aK + kk * 2048, C::kSubBoxBytes),
+                           idesc_acc, (n > 0) || (kk > 0));
+                mma_commit(&bars->st_empty[st]);
+                if (n == n_steps - 1) mma_commit(&bars->acc_full);
+            }
+            if (bars->abort_flag != 0) {
+                mma_commit(&bars->drain);
+                mbar_wait_drain(&bars->drain, 0);
+            }
+        }
+        __syncwarp();
+    } else {
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+        const size_t stat_idx = (static_cast<size_t>(b) * geo.H + h) * geo.N + tq0 + row;
+        const float neg_lse2 = -p.lse[stat_idx] * kLog2e;
+        const float Drow = p.Dsum[stat_idx];
+        const float c2 = p.scale_log2;
+        bool ok = true;
+        for (int n = 0; n < n_steps; ++n) {
+            if (!mbar_wait(&bars->s_full[n & 1], (n >> 1) & 1, ctx, kWaitBwdDq + 5)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t tS = t_row + kColS + (n & 1) * kSubTile;
+            const uint32_t tP = t_row + kColP + (n & 1) * kSubTile;
+            // key x of this sub-tile is visible to query row r iff 64 n + x <= 128 i + r
+            const int lim = i * kTile + row - n * kSubTile;  // visible iff x <= lim
+#pragma unroll
+            for (int c = 0; c < kSubTile / 32; ++c) {
+                uint32_t sr[32], pr[32];
+                tmem_ld_32x32(tS + c * 32, sr);
+                tmem_ld_32x32(tP + c * 32, pr);
+                tmem_wait_ld();
+                float ds[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, neg_lse2));
+                    if (c * 32 + e > lim) pe = 0.f;
+                    ds[e] = pe * (__uint_as_float(pr[e]) - Drow);
+                }
+                uint32_t pk[16];
+                pack32(ds, pk);
+                tmem_st_32x16(tS + c * 16, pk);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&bars->p_full[n & 1]);
+        }
+        if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDq + 6)) {
+            tc_fence_after();
+            __nv_bfloat16* dst = p.dq + ((static_cast<size_t>(b) * geo.N + tq0 + row) * geo.H + h) * HD;
+            store_acc_row<HD>(t_row + kColAcc, p.scale, dst);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, C::kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// 3. dK, dV
+// ------------------------------------------------------------------------------------------------
+// Tensor memory columns: dV [0,HD)  dK [128,128+HD)  S^T buffers [256,320) [320,384)
+//                        dP^T buffers [384,448) [448,512)
+//
+// The CTA owns key tile (b, hk, original tokens tk0 .. tk0+127).  For every query head hq that
+// reads KV head hk (shift s): the tile sits at rolled position (tk0 - s) mod N, i.e. in group g at
+// key tile j, and is attended by query sub-tiles (64 rows) 2j .. 2*Tg-1 of that group.
+struct HeadWalk {
+    int s, g, j, n_begin, n_end;
+};
+__device__ __forceinline__ HeadWalk head_walk(const Geometry& geo, int hq, int tk0) {
+    HeadWalk w;
+    w.s = (hq < geo.n_unshifted) ? 0 : geo.shift;
+    const int pos = mod_pos(tk0 - w.s, geo.N);
+    w.g = pos / geo.G;
+    w.j = (pos % geo.G) / kTile;
+    w.n_begin = 2 * w.j;
+    w.n_end = 2 * geo.tiles_per_group;
+    return w;
+}
+
+template <int HD>
+__global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(const __grid_constant__ BwdDkDvParams p) {
+    using C = BwdCfg<HD>;
+    using Bars = BwdBars<C::kStages>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sK = smem;                                // resident: K_j
+    uint8_t* sV = sK + C::kBigTileBytes;               // resident: V_j
+    uint8_t* sStage = sV + C::kBigTileBytes;           // per stage: Q_n then dO_n
+    float* sStat = reinterpret_cast<float*>(sStage + C::kStages * C::kStageBytes);  // per stage: lse[64], D[64]
+    Bars* bars = reinterpret_cast<Bars*>(reinterpret_cast<uint8_t*>(sStat) + C::kStages * 2 * C::kStatBytes);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const Geometry& geo = p.geo;
+    const int rep = geo.H / geo.Hkv;
+
+    // key tile: enumerate in the rolled order of the first query head of the KV head, heaviest
+    // (earliest in the group) first
+    const int Tg = geo.tiles_per_group;
+    const int j0 = static_cast<int>(blockIdx.x % Tg);
+    const int unit = blockIdx.x / Tg;
+    const int g0 = unit % geo.groups;
+    const int hk = (unit / geo.groups) % geo.Hkv;
+    const int b = unit / (geo.groups * geo.Hkv);
+    const int hq0 = hk * rep;
+    const int s0 = (hq0 < geo.n_unshifted) ? 0 : geo.shift;
+    const int tk0 = mod_pos(g0 * geo.G + j0 * kTile + s0, geo.N);
+
+    int total_steps = 0;
+    for (int hq = hq0; hq < hq0 + rep; ++hq) {
+        const HeadWalk w = head_walk(geo, hq, tk0);
+        total_steps += w.n_end - w.n_begin;
+    }
+
+    if (threadIdx.x == 0) {
+        mbar_init(&bars->res_full, 1);
+        mbar_init(&bars->acc_full, 1);
+        mbar_init(&bars->drain, 1);
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(&bars->s_full[x], 1);
+            mbar_init(&bars->p_full[x], 128);
+        }
+        for (int st = 0; st < C::kStages; ++st) {
+            mbar_init(&bars->st_full[st], 1);
+            mbar_init(&bars->st_empty[st], 1);
+        }
+        bars->abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&p.tm_q);
+        tma_prefetch_desc(&p.tm_do);
+        tma_prefetch_desc(&p.tm_k);
+        tma_prefetch_desc(&p.tm_v);
+    }
+    if (warp == 1) {
+        tmem_alloc(&bars->tmem_slot, C::kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = bars->tmem_slot;
+    const WaitCtx ctx{&bars->abort_flag, p.status};
+    constexpr uint32_t kColDV = 0, kColDK = 128, kColS = 256, kColP = 384;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_expect_tx(&bars->res_full, 2 * C::kBigTileBytes);
+            for (int bx = 0; bx < C::kBoxes; ++bx) {
+                tma_load_4d(sK + bx * C::kBigBoxBytes, &p.tm_k, &bars->res_full, bx * 64, hk, tk0, b);
+                tma_load_4d(sV + bx * C::kBigBoxBytes, &p.tm_v, &bars->res_full, bx * 64, hk, tk0, b);
+            }
+            int it = 0;
+            bool ok = true;
+            for (int hq = hq0; ok && hq < hq0 + rep; ++hq) {
+                const HeadWalk w = head_walk(geo, hq, tk0);
+                for (int n = w.n_begin; n < w.n_end; ++n, ++it) {
+                    const int st = it % C::kStages;
+                    const uint32_t ph = (it / C::kStages) & 1;
+                    const int tq0 = mod_pos(w.g * geo.G + n * kSubTile + w.s, geo.N);
+                    if (!mbar_wait(&bars->st_empty[st], ph ^ 1, ctx, kWaitBwdDkDv + 1)) { ok = false; break; }
+                    mbar_expect_tx(&bars->st_full[st], C::kStageBytes + 2 * C::kStatBytes);
+                    uint8_t* sQ = sStage + st * C::kStageBytes;
+                    uint8_t* sDO = sQ + C::kSubTileBytes;
+                    for (int bx = 0; bx < C::kBoxes; ++bx) {
+                        tma_load_4d(sQ + bx * C::kSubBoxBytes, &p.tm_q, &bars->st_full[st], bx * 64, hq, tq0, b);
+                        tma_load_4d(sDO + bx * C::kSubBoxBytes, &p.tm_do, &bars->st_full[st], bx * 64, hq, tq0, b);
+                    }
+                    const size_t stat_idx = (static_cast<size_t>(b) * geo.H + hq) * geo.N + tq0;
+                    bulk_load_1d(sStat + st * 2 * kSubTile, p.lse + stat_idx, C::kStatBytes, &bars->st_full[st]);
+                    bulk_load_1d(sStat + st * 2 * kSubTile + kSubTile, p.Dsum + stat_idx, C::kStatBytes,
+                                 &bars->st_full[st]);
+                }
+            }
+            if (bars->abort_flag != 0) {
+                mbar_wait_drain(&bars->res_full, 0);
+                for (int nn = (it > C::kStages ? it - C::kStages : 0); nn < it; ++nn)
+                    mbar_wait_drain(&bars->st_full[nn % C::kStages], (nn / C::kStages) & 1);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);  // S^T = K Q^T, dP^T = V dO^T
+            constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);       // dV += P^T dO, dK += dS^T Q
+            const uint32_t aK = smem_u32(sK), aV = smem_u32(sV);
+            auto issue_scores = [&](int it) -> bool {
+                const int st = it % C::kStages;
+                if (!mbar_wait(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 2)) return false;
+                tc_fence_after();
+                const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
+                const uint32_t aDO = aQ + C::kSubTileBytes;
+                const uint32_t tS = tmem_base + kColS + (it & 1) * kSubTile;
+                const uint32_t tP = tmem_base + kColP + (it & 1) * kSubTile;
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t offA = (kk >> 2) * C::kBigBoxBytes + (kk & 3) * 32;
+                    const uint32_t offB = (kk >> 2) * C::kSubBoxBytes + (kk & 3) * 32;
+                    mma_ss(tS, desc_k_major(aK + offA), desc_k_major(aQ + offB), idesc_sc, kk > 0);
+                }
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t offA = (kk >> 2) * C::kBigBoxBytes + (kk & 3) * 32;
+                    const uint32_t offB = (kk >> 2) * C::kSubBoxBytes + (kk & 3) * 32;
+                    mma_ss(tP, desc_k_major(aV + offA), desc_k_major(aDO + offB), idesc_sc, kk > 0);
+                }
+                mma_commit(&bars->s_full[it & 1]);
+                return true;
+            };
+            bool ok = mbar_wait(&bars->res_full, 0, ctx, kWaitBwdDkDv + 3);
+            ok = ok && issue_scores(0);
+            for (int it = 0; ok && it < total_steps; ++it) {
+                if (it + 1 < total_steps && !issue_scores(it + 1)) break;
+                if (!mbar_wait(&bars->p_full[it & 1], (it >> 1) & 1, ctx, kWaitBwdDkDv + 4)) break;
+                tc_fence_after();
+                const int st = it % C::kStages;
+                const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
+                const uint32_t aDO = aQ + C::kSubTileBytes;
+                const uint32_t tPt = tmem_base + kColS + (it & 1) * kSubTile;   // bf16 P^T over the S^T buffer
+                const uint32_t tdSt = tmem_base + kColP + (it & 1) * kSubTile;  // bf16 dS^T over the dP^T buffer
+#pragma unroll
+                for (int kk = 0; kk < kSubTile / 16; ++kk)
+                    mma_ts(tmem_base + kColDV, tPt + kk * 8, desc_mn_major(aDO + kk * 2048, C::kSubBoxBytes),
+                           idesc_acc, (it > 0) || (kk > 0));
+#pragma unroll
+                for (int kk = 0; kk < kSubTile / 16; ++kk)
+                    mma_ts(tmem_base + kColDK, tdSt + kk * 8, desc_mn_major(aQ + kk * 2048, C::kSubBoxBytes),
+                           idesc_acc, (it > 0) || (kk > 0));
+                mma_commit(&bars->st_empty[st]);
+                if (it == total_steps - 1) mma_commit(&bars->acc_full);
+            }
+            if (bars->abort_flag != 0) {
+                mma_commit(&bars->drain);
+                mbar_wait_drain(&bars->drain, 0);
+            }
+        }
+        __syncwarp();
+    } else {
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;  // key row of the tile owned by this thread
+        const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+        const float c2 = p.scale_log2;
+        bool ok = true;
+        int it = 0;
+        for (int hq = hq0; ok && hq < hq0 + rep; ++hq) {
+            const HeadWalk w = head_walk(geo, hq, tk0);
+            for (int n = w.n_begin; n < w.n_end; ++n, ++it) {
+                const int st = it % C::kStages;
+                // the statistics of this step travel with its stage
+                if (!mbar_wait(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 5)) { ok = false; break; }
+                if (!mbar_wait(&bars->s_full[it & 1], (it >> 1) & 1, ctx, kWaitBwdDkDv + 6)) { ok = false; break; }
+                tc_fence_after();
+                const float4* lse4 = reinterpret_cast<const float4*>(sStat + st * 2 * kSubTile);
+                const float4* d4 = lse4 + kSubTile / 4;
+                const uint32_t tS = t_row + kColS + (it & 1) * kSubTile;
+                const uint32_t tP = t_row + kColP + (it & 1) * kSubTile;
+                // query x of this sub-tile sees key row r iff 128 j + r <= 64 n + x
+                const int lim = w.j * kTile + row - n * kSubTile;  // visible iff x >= lim
+#pragma unroll
+                for (int c = 0; c < kSubTile / 32; ++c) {
+                    uint32_t sr[32], pr[32];
+                    tmem_ld_32x32(tS + c * 32, sr);
+                    tmem_ld_32x32(tP + c * 32, pr);
+                    tmem_wait_ld();
+                    float pt[32], ds[32];
+#pragma unroll
+                    for (int e4 = 0; e4 < 8; ++e4) {
+                        const float4 l = lse4[c * 8 + e4];
+                        const float4 dd = d4[c * 8 + e4];
+                        const float lv[4] = {l.x, l.y, l.z, l.w};
+                        const float dv[4] = {dd.x, dd.y, dd.z, dd.w};
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int e = e4 * 4 + u;
+                            float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, -lv[u] * kLog2e));
+                            if (c * 32 + e < lim) pe = 0.f;
+                            pt[e] = pe;
+                            ds[e] = pe * (__uint_as_float(pr[e]) - dv[u]);
+                        }
+                    }
+                    uint32_t pk[16];
+                    pack32(pt, pk);
+                    tmem_st_32x16(tS + c * 16, pk);
+                    pack32(ds, pk);
+                    tmem_st_32x16(tP + c * 16, pk);
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(&bars->p_full[it & 1]);
+            }
+        }
+        if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDkDv + 7)) {
+            tc_fence_after();
+            const size_t out_row = ((static_cast<size_t>(b) * geo.N + tk0 + row) * geo.Hkv + hk) * HD;
+            store_acc_row<HD>(t_row + kColDV, 1.0f, p.dv + out_row);
+            store_acc_row<HD>(t_row + kColDK, p.scale, p.dk + out_row);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, C::kTmemCols);
+    }
+}
+
+}  // namespace
+
+cudaError_t configure_bwd() {
+    cudaError_t e;
+    e = cudaFuncSetAttribute(s2a_bwd_dq_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(s2a_bwd_dq_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<128>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(s2a_bwd_dkdv_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(s2a_bwd_dkdv_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                BwdCfg<128>::kSmemBytes);
+}
+
+cudaError_t launch_bwd_preprocess(const PreParams& p, int d, cudaStream_t stream) {
+    const long long threads = static_cast<long long>(p.B) * p.N * p.H * (d / 8);
+    const unsigned grid = static_cast<unsigned>((threads + 255) / 256);
+    if (d == 64) s2a_bwd_preprocess_kernel<64><<<grid, 256, 0, stream>>>(p);
+    else s2a_bwd_preprocess_kernel<128><<<grid, 256, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_bwd_dq(const BwdDqParams& p, int d, cudaStream_t stream) {
+    const Geometry& g = p.geo;
+    const unsigned grid = static_cast<unsigned>(static_cast<long long>(g.B) * g.H * g.groups * g.tiles_per_group);
+    if (d == 64) s2a_bwd_dq_kernel<64><<<grid, BwdCfg<64>::kThreads, BwdCfg<64>::kSmemBytes, stream>>>(p);
+    else s2a_bwd_dq_kernel<128><<<grid, BwdCfg<128>::kThreads, BwdCfg<128>::kSmemBytes, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_bwd_dkdv(const BwdDkDvParams& p, int d, cudaStream_t stream) {
+    const Geometry& g = p.geo;
+    const unsigned grid = static_cast<unsigned>(static_cast<long long>(g.B) * g.Hkv * g.groups * g.tiles_per_group);
+    if (d == 64) s2a_bwd_dkdv_kernel<64><<<grid, BwdCfg<64>::kThreads, BwdCfg<64>::kSmemBytes, stream>>>(p);
+    else s2a_bwd_dkdv_kernel<128><<<grid, BwdCfg<128>::kThreads, BwdCfg<128>::kSmemBytes, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace s2a

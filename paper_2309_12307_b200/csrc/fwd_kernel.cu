@@ -63,22 +63,22 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
     const int lane = threadIdx.x & 31;
 
     // ---- which tile: heaviest query tiles of a group first, groups of one head adjacent -------
-    const int Tg = p.tiles_per_group;
+    const int Tg = p.geo.tiles_per_group;
     const int it = blockIdx.x % Tg;
     const int unit = blockIdx.x / Tg;
     const int i = Tg - 1 - it;                 // query tile inside the group
-    const int g = unit % p.groups;
-    const int h = (unit / p.groups) % p.H;
-    const int b = unit / (p.groups * p.H);
-    const int hk = h / (p.H / p.Hkv);
-    const int s = (h < p.n_unshifted) ? 0 : p.shift;
+    const int g = unit % p.geo.groups;
+    const int h = (unit / p.geo.groups) % p.geo.H;
+    const int b = unit / (p.geo.groups * p.geo.H);
+    const int hk = h / (p.geo.H / p.geo.Hkv);
+    const int s = (h < p.geo.n_unshifted) ? 0 : p.geo.shift;
     const int n_kv = i + 1;                    // causal: key tiles 0..i of the same group
     // original token of rolled position x:  (x + s) mod N
     auto orig_token = [&](int rolled) {
-        int t = (rolled + s) % p.N;
-        return t < 0 ? t + p.N : t;
+        int t = (rolled + s) % p.geo.N;
+        return t < 0 ? t + p.geo.N : t;
     };
-    const int tq0 = orig_token(g * p.G + i * kTile);
+    const int tq0 = orig_token(g * p.geo.G + i * kTile);
 
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
@@ -118,7 +118,7 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
             for (; j < n_kv; ++j) {
                 const int st = j % C::kStages;
                 const uint32_t ph = (j / C::kStages) & 1;
-                const int tk0 = orig_token(g * p.G + j * kTile);
+                const int tk0 = orig_token(g * p.geo.G + j * kTile);
                 if (!mbar_wait(k_empty + st, ph ^ 1, ctx, kWaitFwd + 1)) break;
                 mbar_expect_tx(k_full + st, C::kTileBytes);
                 for (int bx = 0; bx < C::kBoxes; ++bx)
@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
             tc_fence_after();
             const float inv_l = 1.0f / l;
             const int t = tq0 + row;
-            __nv_bfloat16* orow = p.o + ((static_cast<size_t>(b) * p.N + t) * p.H + h) * HD;
+            __nv_bfloat16* orow = p.o + ((static_cast<size_t>(b) * p.geo.N + t) * p.geo.H + h) * HD;
 #pragma unroll
             for (int c = 0; c < HD / 32; ++c) {
                 uint32_t oreg[32];
@@ -270,7 +270,7 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
                 }
             }
             // natural-log sum-exp of the scaled scores
-            p.lse[(static_cast<size_t>(b) * p.H + h) * p.N + t] = (m_used + log2f(l)) * 0.6931471805599453f;
+            p.lse[(static_cast<size_t>(b) * p.geo.H + h) * p.geo.N + t] = (m_used + log2f(l)) * 0.6931471805599453f;
         }
     }
 
@@ -294,7 +294,7 @@ cudaError_t configure_fwd() {
 }
 
 cudaError_t launch_fwd(const FwdParams& p, int d, cudaStream_t stream) {
-    const long long n_cta = static_cast<long long>(p.B) * p.H * p.groups * p.tiles_per_group;
+    const long long n_cta = static_cast<long long>(p.geo.B) * p.geo.H * p.geo.groups * p.geo.tiles_per_group;
     const dim3 grid(static_cast<unsigned>(n_cta));
     if (d == 64) {
         s2a_fwd_kernel<64><<<grid, FwdCfg<64>::kThreads, FwdCfg<64>::kSmemBytes, stream>>>(p);

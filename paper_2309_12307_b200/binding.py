@@ -1,0 +1,193 @@
+"""Python binding of the C-ABI in include/s2a.h (ctypes; argument marshalling only).
+
+torch is used for device memory and streams.  Every step of the operator runs in the CUDA
+library; there is no fallback: if libs2a.so is missing or a call fails, an exception is raised.
+Operation: S2-Attn, Algorithm 1 / Section 3.2 of the LongLoRA paper (see include/s2a.h).
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libs2a.so")
+
+S2A_OK = 0
+S2A_ERR_INVALID_ARG = -1
+S2A_ERR_UNSUPPORTED = -2
+S2A_ERR_CUDA = -3
+S2A_ERR_TIMEOUT = -4
+
+EXPORTS = [
+    "s2a_fwd", "s2a_bwd", "s2a_bwd_workspace_bytes", "s2a_fwd_ex", "s2a_bwd_ex", "s2a_fwd_bwd_host",
+    "s2a_device_status", "s2a_status_string", "s2a_last_cuda_error", "s2a_version",
+]
+
+_lib = None
+
+
+class S2AError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} (status {status}, cuda error {last_cuda_error()})")
+
+
+def load() -> ctypes.CDLL:
+    """Load libs2a.so (built by paper_2309_12307_b200/build.py).  Raises if it is not there."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2309_12307_b200.build` (needs nvcc)")
+    lib = ctypes.CDLL(LIB_PATH)
+    P, I, F, Z = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.s2a_fwd.argtypes = [P, P, P, P, P, I, I, I, I, I, I, P]
+    lib.s2a_fwd.restype = I
+    lib.s2a_bwd.argtypes = [P, P, P, P, P, P, P, P, P, I, I, I, I, I, I, P, Z, P]
+    lib.s2a_bwd.restype = I
+    lib.s2a_fwd_ex.argtypes = [P, P, P, P, P, I, I, I, I, I, I, F, I, I, P]
+    lib.s2a_fwd_ex.restype = I
+    lib.s2a_bwd_ex.argtypes = [P, P, P, P, P, P, P, P, P, I, I, I, I, I, I, F, I, I, P, Z, P]
+    lib.s2a_bwd_ex.restype = I
+    lib.s2a_bwd_workspace_bytes.argtypes = [I, I, I, I, I, I]
+    lib.s2a_bwd_workspace_bytes.restype = Z
+    lib.s2a_fwd_bwd_host.argtypes = [P] * 18 + [I] * 6 + [P, Z, P]
+    lib.s2a_fwd_bwd_host.restype = I
+    lib.s2a_device_status.argtypes = [ctypes.POINTER(I)]
+    lib.s2a_device_status.restype = I
+    lib.s2a_status_string.argtypes = [I]
+    lib.s2a_status_string.restype = ctypes.c_char_p
+    lib.s2a_last_cuda_error.restype = I
+    lib.s2a_version.restype = I
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load().s2a_status_string(int(status)).decode()
+
+
+def last_cuda_error() -> int:
+    return int(load().s2a_last_cuda_error())
+
+
+def version() -> int:
+    return int(load().s2a_version())
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != S2A_OK:
+        raise S2AError(rc, what)
+
+
+def _dims(q: torch.Tensor, k: torch.Tensor):
+    B, N, H, d = q.shape
+    return B, N, H, k.shape[2], d
+
+
+def _require(t: torch.Tensor, dtype, name: str):
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise ValueError(f"{name} must be a contiguous CUDA tensor of dtype {dtype}")
+
+
+def bwd_workspace_bytes(B, N, H, Hkv, d, G) -> int:
+    return int(load().s2a_bwd_workspace_bytes(B, N, H, Hkv, d, G))
+
+
+def s2a_fwd(q, k, v, G, o=None, lse=None, stream=None):
+    """o [B,N,H,d] bf16 and lse [B,H,N] fp32 of S2-Attn (second half of the heads shifted by G/2)."""
+    B, N, H, Hkv, d = _dims(q, k)
+    for t, n in ((q, "q"), (k, "k"), (v, "v")):
+        _require(t, torch.bfloat16, n)
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device)
+    _require(o, torch.bfloat16, "o")
+    _require(lse, torch.float32, "lse")
+    rc = load().s2a_fwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), B, N, H, Hkv, d, G,
+                        _stream_ptr(stream))
+    _check(rc, "s2a_fwd")
+    return o, lse
+
+
+def s2a_bwd(q, k, v, o, lse, dO, G, dq=None, dk=None, dv=None, workspace=None, stream=None):
+    """dq, dk, dv (bf16) of sum(o * dO)."""
+    B, N, H, Hkv, d = _dims(q, k)
+    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (dO, "dO")):
+        _require(t, torch.bfloat16, n)
+    _require(lse, torch.float32, "lse")
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(v) if dv is None else dv
+    need = bwd_workspace_bytes(B, N, H, Hkv, d, G)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    rc = load().s2a_bwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), dO.data_ptr(),
+                        dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, N, H, Hkv, d, G, workspace.data_ptr(),
+                        workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    _check(rc, "s2a_bwd")
+    return dq, dk, dv
+
+
+def s2a_fwd_ex(q, k, v, G, scale=None, n_unshifted=None, shift=None, o=None, lse=None, stream=None):
+    """Generalised forward: heads [0, n_unshifted) unshifted, the rest rolled by -shift tokens."""
+    B, N, H, Hkv, d = _dims(q, k)
+    scale = 1.0 / math.sqrt(d) if scale is None else scale
+    n_unshifted = H // 2 if n_unshifted is None else n_unshifted
+    shift = G // 2 if shift is None else shift
+    o = torch.empty_like(q) if o is None else o
+    lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if lse is None else lse
+    rc = load().s2a_fwd_ex(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), B, N, H, Hkv, d, G,
+                           scale, n_unshifted, shift, _stream_ptr(stream))
+    _check(rc, "s2a_fwd_ex")
+    return o, lse
+
+
+def s2a_bwd_ex(q, k, v, o, lse, dO, G, scale=None, n_unshifted=None, shift=None, workspace=None, stream=None):
+    B, N, H, Hkv, d = _dims(q, k)
+    scale = 1.0 / math.sqrt(d) if scale is None else scale
+    n_unshifted = H // 2 if n_unshifted is None else n_unshifted
+    shift = G // 2 if shift is None else shift
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    need = bwd_workspace_bytes(B, N, H, Hkv, d, G)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    rc = load().s2a_bwd_ex(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), dO.data_ptr(),
+                           dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, N, H, Hkv, d, G, scale, n_unshifted, shift,
+                           workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    _check(rc, "s2a_bwd_ex")
+    return dq, dk, dv
+
+
+def s2a_fwd_bwd_host(host_in, host_out, dev, G, workspace, stream=None):
+    """Forward+backward from pinned host tensors.
+
+    host_in  = (q, k, v, dO) CPU bf16 tensors; host_out = (o, lse, dq, dk, dv) CPU tensors to fill;
+    dev      = (q, k, v, dO, o, lse, dq, dk, dv) device buffers of the same shapes.
+    Work is only enqueued: synchronise the stream before reading host_out.
+    """
+    hq, hk, hv, hdo = host_in
+    ho, hlse, hdq, hdk, hdv = host_out
+    B, N, H, Hkv, d = _dims(hq, hk)
+    ptrs = [t.data_ptr() for t in (hq, hk, hv, hdo, ho, hlse, hdq, hdk, hdv)] + [t.data_ptr() for t in dev]
+    rc = load().s2a_fwd_bwd_host(*ptrs, B, N, H, Hkv, d, G, workspace.data_ptr(),
+                                 workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    _check(rc, "s2a_fwd_bwd_host")
+
+
+def device_status():
+    """(status, where): S2A_OK, or S2A_ERR_TIMEOUT with the code of the wait that expired."""
+    where = ctypes.c_int(0)
+    rc = load().s2a_device_status(ctypes.byref(where))
+    return int(rc), int(where.value)

@@ -147,6 +147,13 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+
+    // A bounded wait that expired earlier (in any kernel) leaves the status word set: later CTAs
+    // then return at once instead of each running into its own time limit.
+    __shared__ int s_poisoned;
+    if (threadIdx.x == 0) s_poisoned = *reinterpret_cast<volatile int*>(p.status);
+    __syncthreads();
+    if (s_poisoned != 0) return;
     const Geometry& geo = p.geo;
 
     const int Tg = geo.tiles_per_group;
@@ -358,6 +365,13 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+
+    // A bounded wait that expired earlier (in any kernel) leaves the status word set: later CTAs
+    // then return at once instead of each running into its own time limit.
+    __shared__ int s_poisoned;
+    if (threadIdx.x == 0) s_poisoned = *reinterpret_cast<volatile int*>(p.status);
+    __syncthreads();
+    if (s_poisoned != 0) return;
     const Geometry& geo = p.geo;
     const int rep = geo.H / geo.Hkv;
 

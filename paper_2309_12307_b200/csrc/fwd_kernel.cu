@@ -62,6 +62,13 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
+    // A bounded wait that expired earlier (in any kernel) leaves the status word set: later CTAs
+    // then return at once instead of each running into its own time limit.
+    __shared__ int s_poisoned;
+    if (threadIdx.x == 0) s_poisoned = *reinterpret_cast<volatile int*>(p.status);
+    __syncthreads();
+    if (s_poisoned != 0) return;
+
     // ---- which tile: heaviest query tiles of a group first, groups of one head adjacent -------
     const int Tg = p.geo.tiles_per_group;
     const int it = blockIdx.x % Tg;

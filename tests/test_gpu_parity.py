@@ -1,0 +1,234 @@
+"""Parity of the CUDA path (through the C-ABI) against the CPU fp64 oracle, element by element on
+small seeded inputs and on sampled rows at the benchmark's full sizes.
+
+Tolerances (bf16 inputs, fp32 accumulation, bf16 outputs): max abs error 2e-2 on o, relative L2
+error 1e-2 on dq, dk, dv; lse (fp32) within 2e-3.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import s2a_oracle as orc
+from paper_2309_12307_b200.inputs import WORKLOADS, make_inputs
+
+pytestmark = pytest.mark.gpu
+
+O_ATOL = 2e-2
+GRAD_REL_L2 = 1e-2
+LSE_ATOL = 2e-3
+
+
+@pytest.fixture(scope="module")
+def s2a():
+    from paper_2309_12307_b200 import binding
+
+    binding.load()
+    return binding
+
+
+def rel_l2(got, want):
+    got = np.asarray(got, dtype=np.float64)
+    return float(np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30))
+
+
+def run_gpu(s2a, q, k, v, dO, G, **ex):
+    dev = torch.device("cuda:0")
+    qd, kd, vd, dOd = (x.to(dev) for x in (q, k, v, dO))
+    if ex:
+        o, lse = s2a.s2a_fwd_ex(qd, kd, vd, G, **ex)
+        dq, dk, dv = s2a.s2a_bwd_ex(qd, kd, vd, o, lse, dOd, G, **ex)
+    else:
+        o, lse = s2a.s2a_fwd(qd, kd, vd, G)
+        dq, dk, dv = s2a.s2a_bwd(qd, kd, vd, o, lse, dOd, G)
+    torch.cuda.synchronize()
+    rc, where = s2a.device_status()
+    assert rc == 0, f"device status {rc} at wait {where}"
+    return tuple(x.float().cpu().numpy().astype(np.float64) for x in (o, lse, dq, dk, dv))
+
+
+SMALL = [
+    # B, N, G, H, Hkv, d      several tiles per group, wrapped groups, GQA ratios 1/2/4/8
+    (1, 1024, 256, 4, 4, 64),     # the tiny benchmark configuration
+    (1, 512, 256, 2, 2, 128),
+    (2, 1024, 512, 4, 2, 128),
+    (1, 1536, 768, 8, 2, 64),     # group = 6 tiles, not a power of two
+    (1, 1024, 1024, 2, 2, 128),   # single group: the shifted head wraps the whole sequence
+    (2, 512, 256, 8, 1, 128),     # one KV head shared by shifted and unshifted query heads
+    (1, 2048, 1024, 16, 2, 64),   # GQA ratio 8
+]
+
+
+@pytest.mark.parametrize("B,N,G,H,Hkv,d", SMALL)
+def test_small_shapes_match_oracle_everywhere(s2a, B, N, G, H, Hkv, d):
+    q, k, v, dO = make_inputs(B, N, H, Hkv, d, seed=0)
+    o, lse, dq, dk, dv = run_gpu(s2a, q, k, v, dO, G)
+    o_ref, lse_ref = orc.fwd(q, k, v, G)
+    dq_ref, dk_ref, dv_ref = orc.bwd(q, k, v, dO, G)
+    assert np.abs(o - o_ref).max() <= O_ATOL
+    assert np.abs(lse - lse_ref).max() <= LSE_ATOL
+    assert rel_l2(dq, dq_ref) <= GRAD_REL_L2
+    assert rel_l2(dk, dk_ref) <= GRAD_REL_L2
+    assert rel_l2(dv, dv_ref) <= GRAD_REL_L2
+    # per-head slices too, so that one bad head cannot hide in the aggregate
+    for h in range(H):
+        assert rel_l2(dq[:, :, h], dq_ref[:, :, h]) <= GRAD_REL_L2, h
+    for hk in range(Hkv):
+        assert rel_l2(dk[:, :, hk], dk_ref[:, :, hk]) <= GRAD_REL_L2, hk
+        assert rel_l2(dv[:, :, hk], dv_ref[:, :, hk]) <= GRAD_REL_L2, hk
+
+
+def test_generalised_shift_and_head_split(s2a):
+    """Pattern 1 only, pattern 2 only, full causal attention (G = N, nothing shifted), and a
+    custom scale all match the oracle given the same parameters."""
+    B, N, G, H, Hkv, d = 1, 1024, 512, 4, 2, 64
+    q, k, v, dO = make_inputs(B, N, H, Hkv, d, seed=1)
+    cases = [
+        dict(n_unshifted=H, shift=0),
+        dict(n_unshifted=0, shift=G // 2),
+        dict(n_unshifted=1, shift=128, scale=0.2),
+        dict(n_unshifted=2, shift=-(G // 2)),
+    ]
+    for ex in cases:
+        o, lse, dq, dk, dv = run_gpu(s2a, q, k, v, dO, G, **ex)
+        o_ref, lse_ref = orc.fwd(q, k, v, G, **ex)
+        dq_ref, dk_ref, dv_ref = orc.bwd(q, k, v, dO, G, **ex)
+        assert np.abs(o - o_ref).max() <= O_ATOL, ex
+        assert np.abs(lse - lse_ref).max() <= LSE_ATOL, ex
+        for got, want in ((dq, dq_ref), (dk, dk_ref), (dv, dv_ref)):
+            assert rel_l2(got, want) <= GRAD_REL_L2, ex
+    # full causal attention
+    o, lse, dq, dk, dv = run_gpu(s2a, q, k, v, dO, N, n_unshifted=H, shift=0)
+    o_ref, _ = orc.fwd(q, k, v, N, n_unshifted=H, shift=0)
+    assert np.abs(o - o_ref).max() <= O_ATOL
+
+
+def test_outputs_are_deterministic_and_fully_written(s2a):
+    B, N, G, H, Hkv, d = 1, 1024, 256, 4, 2, 128
+    q, k, v, dO = (x.cuda() for x in make_inputs(B, N, H, Hkv, d, seed=2))
+    outs = []
+    for _ in range(2):
+        o = torch.full_like(q, float("nan"))
+        lse = torch.full((B, H, N), float("nan"), device="cuda")
+        s2a.s2a_fwd(q, k, v, G, o=o, lse=lse)
+        dq, dk, dv = (torch.full_like(x, float("nan")) for x in (q, k, v))
+        s2a.s2a_bwd(q, k, v, o, lse, dO, G, dq=dq, dk=dk, dv=dv)
+        torch.cuda.synchronize()
+        outs.append((o, lse, dq, dk, dv))
+    for a, b in zip(*outs):
+        assert not torch.isnan(a).any()
+        assert torch.equal(a, b)
+
+
+def test_guard_bands_stay_intact(s2a):
+    """Outputs sit inside larger buffers filled with a sentinel; nothing outside them may change."""
+    B, N, G, H, Hkv, d = 1, 512, 256, 2, 2, 64
+    q, k, v, dO = (x.cuda() for x in make_inputs(B, N, H, Hkv, d, seed=3))
+    pad = 1024  # elements, keeps 16-byte alignment
+
+    def guarded(shape, dtype):
+        n = int(np.prod(shape))
+        buf = torch.full((n + 2 * pad,), 7.0, dtype=dtype, device="cuda")
+        return buf, buf[pad:pad + n].view(shape)
+
+    bo, o = guarded(q.shape, torch.bfloat16)
+    bl, lse = guarded((B, H, N), torch.float32)
+    bq, dq = guarded(q.shape, torch.bfloat16)
+    bk, dk = guarded(k.shape, torch.bfloat16)
+    bv, dv = guarded(v.shape, torch.bfloat16)
+    s2a.s2a_fwd(q, k, v, G, o=o, lse=lse)
+    s2a.s2a_bwd(q, k, v, o, lse, dO, G, dq=dq, dk=dk, dv=dv)
+    torch.cuda.synchronize()
+    for buf in (bo, bl, bq, bk, bv):
+        assert (buf[:pad] == 7.0).all() and (buf[-pad:] == 7.0).all()
+
+
+def test_runtime_rejections_on_device(s2a):
+    q, k, v, dO = (x.cuda() for x in make_inputs(1, 512, 2, 2, 64, seed=4))
+    with pytest.raises(s2a.S2AError) as e:
+        s2a.s2a_fwd(q, k, v, 128)          # G/2 is not a whole tile
+    assert e.value.status == s2a.S2A_ERR_UNSUPPORTED
+    with pytest.raises(s2a.S2AError) as e:
+        s2a.s2a_fwd(q, k, v, 384)          # N % G
+    assert e.value.status == s2a.S2A_ERR_INVALID_ARG
+    o, lse = s2a.s2a_fwd(q, k, v, 256)
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(s2a.S2AError) as e:
+        s2a.s2a_bwd(q, k, v, o, lse, dO, 256, workspace=small)
+    assert e.value.status == s2a.S2A_ERR_INVALID_ARG
+
+
+# ------------------------------------------------------------------------------------------------
+# full benchmark sizes: sampled rows against the oracle + properties that hold at any size
+# ------------------------------------------------------------------------------------------------
+def _sample_rows(w, kv_tail):
+    N, G, H, Hkv = w.N, w.G, w.H, w.Hkv
+    rep = H // Hkv
+    rng = np.random.default_rng(0)
+    toks = {0, 1, 127, 128, G // 2 - 1, G // 2, G - 1, G, N - G // 2 - 1, N - G // 2, N - 1}
+    toks |= set(int(t) for t in rng.integers(0, N, size=6))
+    heads = sorted({0, H // 2 - 1, H // 2, H - 1})
+    q_rows = [(0, h, t) for h in heads for t in sorted(toks)]
+    # key rows near the end of their group (few queries attend them, so the oracle stays fast):
+    # an unshifted KV head, and a shifted one in its wrapped last group and in an interior group
+    kv_rows = []
+    offs = sorted({1, 2, 64, 65, 128, 129, kv_tail - 1, kv_tail})
+    for off in offs:
+        kv_rows.append((0, 0, G - off))                       # unshifted, group 0
+        kv_rows.append((0, 0, N - off))                       # unshifted, last group
+        kv_rows.append((0, Hkv - 1, (G // 2 - off) % N))      # shifted: end of the wrapped group
+        kv_rows.append((0, Hkv - 1, G + G // 2 - off))        # shifted: end of group 0
+    assert all(h // rep < Hkv for _, h, _ in q_rows)
+    return q_rows, kv_rows
+
+
+FULL = [("llama2_7b_8k", 2048), ("llama2_7b_32k", 1500), ("llama2_70b_32k_gqa", 600), ("llama2_7b_100k", 700)]
+
+
+@pytest.mark.parametrize("name,kv_tail", FULL)
+def test_benchmark_sizes_sampled_rows_and_properties(s2a, name, kv_tail):
+    w = WORKLOADS[name]
+    q, k, v, dO = make_inputs(w.B, w.N, w.H, w.Hkv, w.d, seed=0)
+    dev = torch.device("cuda:0")
+    qd, kd, vd, dOd = (x.to(dev) for x in (q, k, v, dO))
+    o, lse = s2a.s2a_fwd(qd, kd, vd, w.G)
+    dq, dk, dv = s2a.s2a_bwd(qd, kd, vd, o, lse, dOd, w.G)
+    torch.cuda.synchronize()
+    rc, where = s2a.device_status()
+    assert rc == 0, (rc, where)
+
+    q_rows, kv_rows = _sample_rows(w, kv_tail)
+    o_ref, lse_ref = orc.fwd(q, k, v, w.G, rows=q_rows)
+    dq_ref, dk_ref, dv_ref = orc.bwd(q, k, v, dO, w.G, q_rows=q_rows, kv_rows=kv_rows)
+    qi = torch.tensor(q_rows, device=dev)
+    ki = torch.tensor(kv_rows, device=dev)
+    o_s = o[qi[:, 0], qi[:, 2], qi[:, 1]].double().cpu().numpy()
+    lse_s = lse[qi[:, 0], qi[:, 1], qi[:, 2]].double().cpu().numpy()
+    dq_s = dq[qi[:, 0], qi[:, 2], qi[:, 1]].double().cpu().numpy()
+    dk_s = dk[ki[:, 0], ki[:, 2], ki[:, 1]].double().cpu().numpy()
+    dv_s = dv[ki[:, 0], ki[:, 2], ki[:, 1]].double().cpu().numpy()
+    assert np.abs(o_s - o_ref).max() <= O_ATOL
+    assert np.abs(lse_s - lse_ref).max() <= LSE_ATOL
+    assert rel_l2(dq_s, dq_ref) <= GRAD_REL_L2
+    assert rel_l2(dk_s, dk_ref) <= GRAD_REL_L2
+    assert rel_l2(dv_s, dv_ref) <= GRAD_REL_L2
+
+    # properties that hold at any size (they touch every tile of every output)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+    rep = w.H // w.Hkv
+    # rows of P sum to one: sum over keys of dV equals the sum over queries of dO, per KV head
+    dv_sum = dv.double().sum(dim=1)                                        # [B, Hkv, d]
+    do_sum = dOd.double().view(w.B, w.N, w.Hkv, rep, w.d).sum(dim=(1, 3))  # [B, Hkv, d]
+    scale_ref = dOd.double().abs().view(w.B, w.N, w.Hkv, rep, w.d).sum(dim=(1, 3))
+    assert ((dv_sum - do_sum).abs() / scale_ref).max().item() < 5e-3
+    # sum over (t, c) of dQ*q equals sum over (t', c) of dK*k per KV head (both are sum of dS*z)
+    lhs = (dq.double() * qd.double()).view(w.B, w.N, w.Hkv, rep, w.d).sum(dim=(1, 3, 4))
+    rhs = (dk.double() * kd.double()).sum(dim=(1, 3))
+    mag = (dq.double() * qd.double()).abs().view(w.B, w.N, w.Hkv, rep, w.d).sum(dim=(1, 3, 4))
+    assert ((lhs - rhs).abs() / mag).max().item() < 5e-3
+    # the first member of every group attends only itself: o = v there
+    for h in (0, w.H - 1):
+        s = 0 if h < w.H // 2 else w.G // 2
+        t_first = torch.tensor([(g * w.G + s) % w.N for g in range(w.N // w.G)], device=dev)
+        assert torch.equal(o[0, t_first, h], vd[0, t_first, h // rep])

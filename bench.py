@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of S2-Attn forward+backward on B200.
+
+    python bench.py --gpus N --steps K --warmup W            # the CUDA library (this repository)
+    python bench.py --impl reference --steps K --warmup W    # the CPU fp64 oracle, as it stands
+
+A step is one forward + backward pass of the whole operator over one synthetic batch of the
+workload (default: Llama2-7B attention shape, N=32768, G=8192, H=Hkv=32, d=128, bf16).  The metric
+is TFLOP/s counting only the causal in-group FLOPs: 14 * d per attended (query, key) pair.
+With more than one GPU every rank runs an independent replica (the operator has no exchange
+step); the value is the sum over ranks divided by the slowest rank's time.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "S2-Attn fwd+bwd TFLOP/s (causal in-group FLOPs)"
+UNIT = "TFLOP/s"
+DEFAULT_WORKLOAD = "llama2_7b_32k"
+FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks: sample nvidia-smi while the timed region runs
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="s2a_clocks_", suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return res
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 8:
+                    continue
+                try:
+                    sm.append(float(parts[1]))
+                    mx.append(float(parts[2]))
+                    power.append(float(parts[3]))
+                except ValueError:
+                    continue
+                for n, val in zip(names, parts[4:8]):
+                    if val.lower().startswith("active"):
+                        reasons.add(n)
+        os.unlink(self.path)
+        if sm:
+            res.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm),
+                       power_w_max=max(power))
+        return res
+
+
+# ------------------------------------------------------------------------------------------------
+# the CPU oracle, timed (never tuned for this): one whole (batch, head, group) unit per step
+# ------------------------------------------------------------------------------------------------
+def oracle_unit_rows(w, which: int):
+    """Rows of one whole unit: step 0 takes the shifted, wrapped last group of the last head, step 1
+    the first group of head 0, and so on alternating through heads."""
+    H, G, N = w.H, w.G, w.N
+    if which % 2 == 0:
+        h = H - 1 - (which // 2) % (H // 2)
+        g, s = N // G - 1, G // 2
+    else:
+        h = (which // 2) % (H // 2)
+        g, s = 0, 0
+    toks = [(g * G + p + s) % N for p in range(G)]
+    rep = H // w.Hkv
+    hk = h // rep
+    # with grouped-query heads the unit is the KV head's group together with all its query heads
+    q_rows = [(0, hq, t) for hq in range(hk * rep, (hk + 1) * rep) for t in toks]
+    kv_rows = [(0, hk, t) for t in toks]
+    return q_rows, kv_rows
+
+
+def time_oracle_steps(w, inputs, steps: int, warmup: int):
+    from oracle import s2a_oracle as orc
+
+    q, k, v, dO = inputs
+    unit_flops = 14 * w.d * (w.G * (w.G + 1) // 2) * (w.H // w.Hkv)
+    times = []
+    for it in range(warmup + steps):
+        q_rows, kv_rows = oracle_unit_rows(w, it)
+        t0 = time.perf_counter()
+        orc.fwd(q, k, v, w.G, rows=q_rows)
+        orc.bwd(q, k, v, dO, w.G, q_rows=q_rows, kv_rows=kv_rows)
+        dt = time.perf_counter() - t0
+        if it >= warmup:
+            times.append(dt)
+    total = sum(times)
+    return unit_flops * steps / total / 1e12, total / steps, orc.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from paper_2309_12307_b200.inputs import WORKLOADS, make_workload_inputs
+
+    w = WORKLOADS[args.workload]
+    inputs = make_workload_inputs(w, seed=0)
+    tflops, sec_per_step, cores = time_oracle_steps(w, inputs, args.steps, args.warmup)
+    sample = (f"each step = forward+backward of one whole (batch, head, group) unit of {w.name} "
+              f"(G={w.G} queries x causal keys, 1/{w.B * w.H * (w.N // w.G)} of the workload), fp64, OpenMP")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tflops, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec_per_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "N": w.N, "G": w.G, "H": w.H, "Hkv": w.Hkv, "d": w.d,
+                   "sample": sample},
+        "cpu_baseline": {"value": tflops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": tflops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA library
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2309_12307_b200 import binding as s2a
+    from paper_2309_12307_b200.inputs import WORKLOADS, make_workload_inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the operator has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    s2a.load()
+
+    w = WORKLOADS[args.workload]
+    B, N, H, Hkv, d, G = w.B, w.N, w.H, w.Hkv, w.d, w.G
+    host_in = make_workload_inputs(w, seed=0)                       # same bits on every rank (replicas)
+    q, k, v, dO = (x.to(dev) for x in host_in)
+    o = torch.empty_like(q)
+    lse = torch.empty((B, H, N), dtype=torch.float32, device=dev)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    ws = torch.empty(max(s2a.bwd_workspace_bytes(B, N, H, Hkv, d, G), 256), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step_plain():
+        s2a.s2a_fwd(q, k, v, G, o=o, lse=lse, stream=stream)
+        s2a.s2a_bwd(q, k, v, o, lse, dO, G, dq=dq, dk=dk, dv=dv, workspace=ws, stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step_plain()
+    barrier()
+    rc, where = s2a.device_status()
+    if rc != 0:
+        raise RuntimeError(f"device status {rc} (wait code {where}) after warm-up")
+
+    # ---- timed region: exactly K steps; the same four launches per step as s2a_fwd + s2a_bwd, with
+    # events between them so that every kernel's duration is measured inside the region
+    names = ["fwd", "bwd_preprocess", "bwd_dkdv", "bwd_dq"]
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(K)]
+    try:
+        smi_index = int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank])
+    except (KeyError, ValueError, IndexError):
+        smi_index = local_rank
+    sampler = ClockSampler(smi_index)
+    barrier()
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    barrier()
+    for i in range(K):
+        ev[i][0].record(stream)
+        s2a.s2a_fwd(q, k, v, G, o=o, lse=lse, stream=stream)
+        ev[i][1].record(stream)
+        for stage in range(3):
+            s2a.s2a_bwd_stage(q, k, v, o, lse, dO, G, dq, dk, dv, ws, stage, stream=stream)
+            ev[i][2 + stage].record(stream)
+    end = torch.cuda.Event(enable_timing=True)
+    end.record(stream)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = ev[0][0].elapsed_time(end)
+    kernel_ms = {n: sum(ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(K)) for j, n in enumerate(names)}
+    rc, where = s2a.device_status()
+    if rc != 0:
+        raise RuntimeError(f"device status {rc} (wait code {where}) in the timed region")
+
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms_max = float(t.item())
+    flops_step = w.flops_fwd_bwd
+    value = world * flops_step * K / (total_ms_max * 1e-3) / 1e12
+
+    # ---- end to end through the host-buffer entry point: pinned host inputs copied in, all outputs
+    # copied back, every step
+    pin = [x.pin_memory() for x in host_in]
+    host_out = [torch.empty(o.shape, dtype=torch.bfloat16).pin_memory(),
+                torch.empty(lse.shape, dtype=torch.float32).pin_memory(),
+                torch.empty(dq.shape, dtype=torch.bfloat16).pin_memory(),
+                torch.empty(dk.shape, dtype=torch.bfloat16).pin_memory(),
+                torch.empty(dv.shape, dtype=torch.bfloat16).pin_memory()]
+    dev_bufs = (q, k, v, dO, o, lse, dq, dk, dv)
+    h2d = sum(x.numel() * x.element_size() for x in pin)
+    d2h = sum(x.numel() * x.element_size() for x in host_out)
+    Ke = max(3, min(K, 10))
+    for _ in range(2):
+        s2a.s2a_fwd_bwd_host(pin, host_out, dev_bufs, G, ws, stream=stream)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(Ke):
+        s2a.s2a_fwd_bwd_host(pin, host_out, dev_bufs, G, ws, stream=stream)
+    e1.record(stream)
+    barrier()
+    te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_value = world * flops_step * Ke / (float(te.item()) * 1e-3) / 1e12
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- roofline of the dominant kernel (tensor-core bound: a dense contraction).  Algorithmic
+    # FLOPs per launch: forward 4 d per pair; dK/dV kernel 8 d per pair (S, dP, dV, dK); dQ kernel
+    # 2 d per pair (its recomputed S and dP are not counted); preprocess: none counted.
+    peaks, peak_src = load_peaks()
+    pairs = w.pairs
+    alg_flops = {"fwd": 4 * d * pairs, "bwd_preprocess": 0, "bwd_dkdv": 8 * d * pairs, "bwd_dq": 2 * d * pairs}
+    exe_flops = {"fwd": 4 * d * pairs, "bwd_preprocess": 0, "bwd_dkdv": 8 * d * pairs, "bwd_dq": 6 * d * pairs}
+    kernels = {}
+    for n in names:
+        ms = kernel_ms[n] / K
+        kernels[n] = {"launches": K, "ms_per_launch": ms, "share": kernel_ms[n] / sum(kernel_ms.values()),
+                      "algorithmic_tflops": alg_flops[n] / (ms * 1e-3) / 1e12 if ms > 0 else None,
+                      "executed_tflops": exe_flops[n] / (ms * 1e-3) / 1e12 if ms > 0 else None}
+    dom = max(names, key=lambda n: kernel_ms[n])
+    peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+    achieved = kernels[dom]["algorithmic_tflops"]
+    roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": None,
+                "peak_source": f"{peak_src} bf16 sustained (burst {peaks.get('bf16_tflops')})",
+                "whole_step_frac": value / world / peak}
+
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        tf, sec, cores = time_oracle_steps(w, host_in, steps=2, warmup=0)
+        cpu_baseline = {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"2 whole (batch, head, group) units of {w.name} (the shifted wrapped last group "
+                                  f"of head {H - 1}, the first group of head 0), forward+backward, {sec:.1f} s each"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+        "ms_per_step": total_ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "B": B, "N": N, "G": G, "H": H, "Hkv": Hkv, "d": d,
+                   "l2": "inputs (5 x %.0f MB) larger than L2" % (q.numel() * 2 / 1e6),
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "tokens_per_s": world * B * N * K / (total_ms_max * 1e-3),
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": Ke},
+        "gpu_launches": 4 * K,
+        "roofline": roofline,
+        "kernels": kernels,
+        "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -92,6 +92,18 @@ int s2a_bwd_ex(const void* q, const void* k, const void* v, const void* o, const
                void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * One kernel of s2a_bwd at a time, for profiling and per-kernel timing: same arguments and
+ * semantics as s2a_bwd, but only kernel `stage` is enqueued:
+ *   0 = D = rowsum(dO * o) into the workspace, 1 = dk and dv, 2 = dq.
+ * Stages 1 and 2 read the workspace stage 0 wrote.  Calling stages 0, 1, 2 in order on one stream
+ * is exactly s2a_bwd.
+ */
+int s2a_bwd_stage(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO,
+                  void* dq, void* dk, void* dv,
+                  int B, int N, int H, int Hkv, int d, int G,
+                  void* workspace, size_t workspace_bytes, int stage, void* stream);
+
+/*
  * Forward + backward from HOST buffers (pinned memory recommended): copies q, k, v, dO to the
  * caller's device buffers, runs s2a_fwd and s2a_bwd, and copies o, lse, dq, dk, dv back, all
  * enqueued on `stream`; the caller synchronises the stream before reading the host outputs.

@@ -22,7 +22,7 @@ S2A_ERR_CUDA = -3
 S2A_ERR_TIMEOUT = -4
 
 EXPORTS = [
-    "s2a_fwd", "s2a_bwd", "s2a_bwd_workspace_bytes", "s2a_fwd_ex", "s2a_bwd_ex", "s2a_fwd_bwd_host",
+    "s2a_fwd", "s2a_bwd", "s2a_bwd_workspace_bytes", "s2a_fwd_ex", "s2a_bwd_ex", "s2a_bwd_stage", "s2a_fwd_bwd_host",
     "s2a_device_status", "s2a_status_string", "s2a_last_cuda_error", "s2a_version",
 ]
 
@@ -53,6 +53,8 @@ def load() -> ctypes.CDLL:
     lib.s2a_fwd_ex.restype = I
     lib.s2a_bwd_ex.argtypes = [P, P, P, P, P, P, P, P, P, I, I, I, I, I, I, F, I, I, P, Z, P]
     lib.s2a_bwd_ex.restype = I
+    lib.s2a_bwd_stage.argtypes = [P, P, P, P, P, P, P, P, P, I, I, I, I, I, I, P, Z, I, P]
+    lib.s2a_bwd_stage.restype = I
     lib.s2a_bwd_workspace_bytes.argtypes = [I, I, I, I, I, I]
     lib.s2a_bwd_workspace_bytes.restype = Z
     lib.s2a_fwd_bwd_host.argtypes = [P] * 18 + [I] * 6 + [P, Z, P]
@@ -138,6 +140,15 @@ def s2a_bwd(q, k, v, o, lse, dO, G, dq=None, dk=None, dv=None, workspace=None, s
                         workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     _check(rc, "s2a_bwd")
     return dq, dk, dv
+
+
+def s2a_bwd_stage(q, k, v, o, lse, dO, G, dq, dk, dv, workspace, stage, stream=None):
+    """Enqueue one kernel of the backward: 0 = D preprocess, 1 = dk/dv, 2 = dq (profiling aid)."""
+    B, N, H, Hkv, d = _dims(q, k)
+    rc = load().s2a_bwd_stage(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), dO.data_ptr(),
+                              dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, N, H, Hkv, d, G, workspace.data_ptr(),
+                              workspace.numel() * workspace.element_size(), int(stage), _stream_ptr(stream))
+    _check(rc, "s2a_bwd_stage")
 
 
 def s2a_fwd_ex(q, k, v, G, scale=None, n_unshifted=None, shift=None, o=None, lse=None, stream=None):

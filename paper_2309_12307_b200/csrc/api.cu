@@ -173,9 +173,12 @@ size_t s2a_bwd_workspace_bytes(int B, int N, int H, int Hkv, int d, int G) {
     return (bytes + 255) & ~static_cast<size_t>(255);
 }
 
-int s2a_bwd_ex(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO, void* dq,
-               void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, float scale, int n_unshifted,
-               int shift, void* workspace, size_t workspace_bytes, void* stream) {
+namespace {
+enum : unsigned { kStagePre = 1u, kStageDkDv = 2u, kStageDq = 4u, kStageAll = 7u };
+
+int bwd_impl(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO, void* dq,
+             void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, float scale, int n_unshifted, int shift,
+             void* workspace, size_t workspace_bytes, void* stream, unsigned stages) {
     if (!q || !k || !v || !o || !lse || !dO || !dq || !dk || !dv || !workspace) return S2A_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse) || !aligned16(dO) ||
         !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
@@ -214,13 +217,38 @@ int s2a_bwd_ex(const void* q, const void* k, const void* v, const void* o, const
     pp.o = static_cast<const __nv_bfloat16*>(o), pp.dO = static_cast<const __nv_bfloat16*>(dO), pp.Dsum = Dsum;
     pp.B = B, pp.N = N, pp.H = H;
 
-    cudaError_t e = launch_bwd_preprocess(pp, d, st);
-    if (e != cudaSuccess) return cuda_fail(e);
-    e = launch_bwd_dkdv(pk, d, st);
-    if (e != cudaSuccess) return cuda_fail(e);
-    e = launch_bwd_dq(pq, d, st);
-    if (e != cudaSuccess) return cuda_fail(e);
+    cudaError_t e;
+    if (stages & kStagePre) {
+        e = launch_bwd_preprocess(pp, d, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (stages & kStageDkDv) {
+        e = launch_bwd_dkdv(pk, d, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (stages & kStageDq) {
+        e = launch_bwd_dq(pq, d, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
     return S2A_OK;
+}
+}  // namespace
+
+int s2a_bwd_ex(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO, void* dq,
+               void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, float scale, int n_unshifted,
+               int shift, void* workspace, size_t workspace_bytes, void* stream) {
+    return bwd_impl(q, k, v, o, lse, dO, dq, dk, dv, B, N, H, Hkv, d, G, scale, n_unshifted, shift, workspace,
+                    workspace_bytes, stream, kStageAll);
+}
+
+int s2a_bwd_stage(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO,
+                  void* dq, void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, void* workspace,
+                  size_t workspace_bytes, int stage, void* stream) {
+    if (stage < 0 || stage > 2) return S2A_ERR_INVALID_ARG;
+    if (d <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
+    if (G % (2 * kTile) != 0) return (G > 0 && N > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
+    return bwd_impl(q, k, v, o, lse, dO, dq, dk, dv, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2,
+                    G / 2, workspace, workspace_bytes, stream, 1u << stage);
 }
 
 int s2a_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO, void* dq,

@@ -52,6 +52,7 @@ class ClockSampler:
         self.gpu_index = gpu_index
         self.proc = None
         self.path = None
+        self.skip_bytes = 0
 
     def start(self):
         try:
@@ -60,9 +61,16 @@ class ClockSampler:
             self.out = open(self.path, "w")
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=self.out, stderr=subprocess.DEVNULL)
+                 "-lms", "50"], stdout=self.out, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
+            return
+        # nvidia-smi needs a moment before its first sample: wait for it (bounded), then forget
+        # what was sampled while idle
+        t0 = time.time()
+        while time.time() - t0 < 5.0 and os.path.getsize(self.path) == 0:
+            time.sleep(0.05)
+        self.skip_bytes = os.path.getsize(self.path)
 
     def stop(self):
         res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
@@ -77,6 +85,7 @@ class ClockSampler:
         sm, mx, reasons, power = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         with open(self.path) as f:
+            f.seek(self.skip_bytes)
             for line in f:
                 parts = [x.strip() for x in line.split(",")]
                 if len(parts) < 8:
@@ -223,7 +232,6 @@ def run_ours(args):
     barrier()
     if rank == 0:
         sampler.start()
-        time.sleep(0.25)
     barrier()
     for i in range(K):
         ev[i][0].record(stream)
@@ -333,8 +341,8 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -107,11 +107,16 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------
-# the CPU oracle, timed (never tuned for this): one whole (batch, head, group) unit per step
+# the CPU oracle, timed as it stands (never tuned for this)
 # ------------------------------------------------------------------------------------------------
-def oracle_unit_rows(w, which: int):
-    """Rows of one whole unit: step 0 takes the shifted, wrapped last group of the last head, step 1
-    the first group of head 0, and so on alternating through heads."""
+# A sample is the tail of one (batch, KV head, group) unit: the query rows (of every query head of
+# the KV head) and the key rows at in-group positions [G - n, G); n = G is the whole unit.
+# FLOPs credited to a sample, so that a whole unit gets exactly 14 d per attended pair:
+#   an o row: 4 d per pair it attends; a dq row: 10 d / 3 per pair; a (dk, dv) row: 20 d / 3 per
+#   pair that attends it  (the 10 d of the backward split evenly over its three outputs).
+def oracle_sample_rows(w, which: int, n: int):
+    """Step 0 takes the shifted, wrapped last group of the last head, step 1 the first group of
+    head 0, and so on alternating through heads."""
     H, G, N = w.H, w.G, w.N
     if which % 2 == 0:
         h = H - 1 - (which // 2) % (H // 2)
@@ -119,31 +124,42 @@ def oracle_unit_rows(w, which: int):
     else:
         h = (which // 2) % (H // 2)
         g, s = 0, 0
-    toks = [(g * G + p + s) % N for p in range(G)]
+    toks = [(g * G + p + s) % N for p in range(G - n, G)]
     rep = H // w.Hkv
     hk = h // rep
-    # with grouped-query heads the unit is the KV head's group together with all its query heads
     q_rows = [(0, hq, t) for hq in range(hk * rep, (hk + 1) * rep) for t in toks]
     kv_rows = [(0, hk, t) for t in toks]
     return q_rows, kv_rows
 
 
-def time_oracle_steps(w, inputs, steps: int, warmup: int):
+def oracle_sample_flops(w, n: int) -> float:
+    rep = w.H // w.Hkv
+    pairs_q = n * w.G - n * (n - 1) // 2      # sum over positions p in [G-n, G) of (p + 1)
+    pairs_kv = n * (n + 1) // 2               # sum over positions p' in [G-n, G) of (G - p')
+    return rep * w.d * (4.0 * pairs_q + 10.0 / 3.0 * pairs_q + 20.0 / 3.0 * pairs_kv)
+
+
+def oracle_run_sample(w, inputs, which: int, n: int) -> float:
     from oracle import s2a_oracle as orc
 
     q, k, v, dO = inputs
-    unit_flops = 14 * w.d * (w.G * (w.G + 1) // 2) * (w.H // w.Hkv)
+    q_rows, kv_rows = oracle_sample_rows(w, which, n)
+    t0 = time.perf_counter()
+    orc.fwd(q, k, v, w.G, rows=q_rows)
+    orc.bwd(q, k, v, dO, w.G, q_rows=q_rows, kv_rows=kv_rows)
+    return time.perf_counter() - t0
+
+
+def time_oracle_steps(w, inputs, steps: int, warmup: int, n: int):
+    from oracle import s2a_oracle as orc
+
     times = []
     for it in range(warmup + steps):
-        q_rows, kv_rows = oracle_unit_rows(w, it)
-        t0 = time.perf_counter()
-        orc.fwd(q, k, v, w.G, rows=q_rows)
-        orc.bwd(q, k, v, dO, w.G, q_rows=q_rows, kv_rows=kv_rows)
-        dt = time.perf_counter() - t0
+        dt = oracle_run_sample(w, inputs, it, n)
         if it >= warmup:
             times.append(dt)
     total = sum(times)
-    return unit_flops * steps / total / 1e12, total / steps, orc.num_threads()
+    return oracle_sample_flops(w, n) * steps / total / 1e12, total / steps, orc.num_threads()
 
 
 def run_reference(args):
@@ -154,15 +170,23 @@ def run_reference(args):
 
     w = WORKLOADS[args.workload]
     inputs = make_workload_inputs(w, seed=0)
-    tflops, sec_per_step, cores = time_oracle_steps(w, inputs, args.steps, args.warmup)
-    sample = (f"each step = forward+backward of one whole (batch, head, group) unit of {w.name} "
-              f"(G={w.G} queries x causal keys, 1/{w.B * w.H * (w.N // w.G)} of the workload), fp64, OpenMP")
+    # size the per-step sample so that all warm-up and timed steps fit in about two minutes
+    n_cal = min(64, w.G)
+    t_cal = oracle_run_sample(w, inputs, 1, n_cal)
+    rate = oracle_sample_flops(w, n_cal) / max(t_cal, 1e-6)           # credited FLOP/s, roughly constant
+    budget = 120.0 / max(args.steps + args.warmup, 1)
+    n = w.G
+    while n > 64 and oracle_sample_flops(w, n) / rate > budget:
+        n //= 2
+    tflops, sec_per_step, cores = time_oracle_steps(w, inputs, args.steps, args.warmup, n)
+    sample = (f"each step = oracle forward+backward of the query rows and key rows at the last {n} of {w.G} "
+              f"in-group positions of one (batch, head, group) unit of {w.name}, fp64, OpenMP; FLOPs credited: "
+              f"4d per pair of an o row, 10d/3 of a dq row, 20d/3 of a dk/dv row")
     line = {
         "impl": "reference", "metric": METRIC, "value": tflops, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec_per_step * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "N": w.N, "G": w.G, "H": w.H, "Hkv": w.Hkv, "d": w.d,
-                   "sample": sample},
+        "config": {"workload": w.name, "B": w.B, "N": w.N, "G": w.G, "H": w.H, "Hkv": w.Hkv, "d": w.d},
         "cpu_baseline": {"value": tflops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": tflops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -311,7 +335,7 @@ def run_ours(args):
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
-        tf, sec, cores = time_oracle_steps(w, host_in, steps=2, warmup=0)
+        tf, sec, cores = time_oracle_steps(w, host_in, steps=2, warmup=0, n=w.G)
         cpu_baseline = {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle",
                         "sample": f"2 whole (batch, head, group) units of {w.name} (the shifted wrapped last group "
                                   f"of head {H - 1}, the first group of head 0), forward+backward, {sec:.1f} s each"}

@@ -44,7 +44,8 @@ typedef enum s2a_status {
     S2A_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, N % G, odd G or H, H % Hkv, misaligned pointer, small workspace */
     S2A_ERR_UNSUPPORTED = -2, /* d not in {64,128}, G not a multiple of 256, device is not sm_100 */
     S2A_ERR_CUDA = -3,        /* a CUDA call failed while enqueuing; see s2a_last_cuda_error() */
-    S2A_ERR_TIMEOUT = -4      /* reported by s2a_device_status(): a bounded device-side wait expired */
+    S2A_ERR_TIMEOUT = -4,     /* reported by s2a_device_status(): a bounded device-side wait expired */
+    S2A_ERR_TOO_LARGE = -5    /* s2a_bwd_noalloc only: B*H*N is more than its built-in scratch holds */
 } s2a_status;
 
 /*
@@ -90,6 +91,41 @@ int s2a_bwd_ex(const void* q, const void* k, const void* v, const void* o, const
                int B, int N, int H, int Hkv, int d, int G,
                float scale, int n_unshifted, int shift,
                void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * s2a_bwd for callers that have no scratch to give.  (The paper has no counterpart to this entry
+ * point; it exists for integration reasons only.)
+ *
+ * Who needs it: code that is not allowed, or not able, to obtain device memory at the moment it
+ * wants gradients -- a plug-in running inside a host application that owns all device memory and
+ * exposes no allocator; a service whose memory budget was handed out in full at start-up; a
+ * latency-critical loop that must not meet the implicit device-wide synchronisation and the
+ * unpredictable cost of cudaMalloc / cudaFree; a component whose rules forbid allocation after
+ * initialisation.  s2a_bwd wants a workspace from such a caller; this variant does not.
+ *
+ * It computes exactly what s2a_bwd computes (same kernels, same results), but keeps
+ * D = rowsum(dO * o) in an array that is part of the library image: 2^20 fp32 values (4 MiB) on
+ * every GPU that loads the library, held until the process exits.  It calls no allocation routine
+ * of any kind.
+ *
+ *   Limit     : B * H * N <= s2a_bwd_noalloc_max_rows() (= 1,048,576; e.g. B=1, H=32, N=32768).
+ *               Larger problems return S2A_ERR_TOO_LARGE and enqueue nothing; use s2a_bwd.
+ *   Set-up    : the first call on each device looks up the array's device address (with that
+ *               device current).  Make that first call outside any stream capture.
+ *   Sharing   : all calls on a device use the same array.  Calls issued to one stream are ordered
+ *               and safe.  Two calls that can run on the GPU at the same time (different streams,
+ *               or different host threads on different streams) overwrite each other's D and
+ *               give wrong gradients: serialise them, or use s2a_bwd with separate workspaces.
+ *   Contents  : the array keeps whatever the previous call left; every value a call reads is
+ *               first rewritten by that same call, so nothing needs clearing in between.
+ * Other arguments, shapes, errors and the meaning of `stream` are those of s2a_bwd.
+ */
+int s2a_bwd_noalloc(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO,
+                    void* dq, void* dk, void* dv,
+                    int B, int N, int H, int Hkv, int d, int G, void* stream);
+
+/* Largest B * H * N that s2a_bwd_noalloc accepts. */
+size_t s2a_bwd_noalloc_max_rows(void);
 
 /*
  * One kernel of s2a_bwd at a time, for profiling and per-kernel timing: same arguments and

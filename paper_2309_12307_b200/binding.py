@@ -20,9 +20,11 @@ S2A_ERR_INVALID_ARG = -1
 S2A_ERR_UNSUPPORTED = -2
 S2A_ERR_CUDA = -3
 S2A_ERR_TIMEOUT = -4
+S2A_ERR_TOO_LARGE = -5
 
 EXPORTS = [
     "s2a_fwd", "s2a_bwd", "s2a_bwd_workspace_bytes", "s2a_fwd_ex", "s2a_bwd_ex", "s2a_bwd_stage", "s2a_fwd_bwd_host",
+    "s2a_bwd_noalloc", "s2a_bwd_noalloc_max_rows",
     "s2a_device_status", "s2a_status_string", "s2a_last_cuda_error", "s2a_version",
 ]
 
@@ -55,6 +57,9 @@ def load() -> ctypes.CDLL:
     lib.s2a_bwd_ex.restype = I
     lib.s2a_bwd_stage.argtypes = [P, P, P, P, P, P, P, P, P, I, I, I, I, I, I, P, Z, I, P]
     lib.s2a_bwd_stage.restype = I
+    lib.s2a_bwd_noalloc.argtypes = [P, P, P, P, P, P, P, P, P, I, I, I, I, I, I, P]
+    lib.s2a_bwd_noalloc.restype = I
+    lib.s2a_bwd_noalloc_max_rows.restype = Z
     lib.s2a_bwd_workspace_bytes.argtypes = [I, I, I, I, I, I]
     lib.s2a_bwd_workspace_bytes.restype = Z
     lib.s2a_fwd_bwd_host.argtypes = [P] * 18 + [I] * 6 + [P, Z, P]
@@ -139,6 +144,25 @@ def s2a_bwd(q, k, v, o, lse, dO, G, dq=None, dk=None, dv=None, workspace=None, s
                         dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, N, H, Hkv, d, G, workspace.data_ptr(),
                         workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     _check(rc, "s2a_bwd")
+    return dq, dk, dv
+
+
+def bwd_noalloc_max_rows() -> int:
+    return int(load().s2a_bwd_noalloc_max_rows())
+
+
+def s2a_bwd_noalloc(q, k, v, o, lse, dO, G, dq, dk, dv, stream=None):
+    """s2a_bwd for callers that cannot supply scratch: D lives in a 4 MiB array inside the library.
+
+    Outputs are written into the dq, dk, dv tensors the caller passes; this wrapper creates no
+    tensor.  B*H*N must not exceed bwd_noalloc_max_rows().  Calls that may overlap on the GPU
+    share the array and must be serialised (see include/s2a.h).
+    """
+    B, N, H, Hkv, d = _dims(q, k)
+    rc = load().s2a_bwd_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(),
+                                dO.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, N, H, Hkv, d, G,
+                                _stream_ptr(stream))
+    _check(rc, "s2a_bwd_noalloc")
     return dq, dk, dv
 
 

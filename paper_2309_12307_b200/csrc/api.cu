@@ -131,6 +131,7 @@ const char* s2a_status_string(int status) {
         case S2A_ERR_UNSUPPORTED: return "unsupported shape or device (need d in {64,128}, G and shift multiples of 128, sm_100)";
         case S2A_ERR_CUDA: return "a CUDA call failed; see s2a_last_cuda_error()";
         case S2A_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case S2A_ERR_TOO_LARGE: return "B*H*N exceeds the built-in scratch of s2a_bwd_noalloc (see s2a_bwd_noalloc_max_rows)";
         default: return "unknown status";
     }
 }
@@ -292,6 +293,56 @@ int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const vo
     if ((e = cudaMemcpyAsync(h_dv, d_dv, nk, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
     return S2A_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Backward without caller-provided scratch
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+// Built-in home for D = rowsum(dO * o) when the caller cannot provide a workspace: 2^20 fp32 rows
+// (4 MiB), which every GPU that loads this library keeps resident until the process exits.
+constexpr size_t kBuiltinScratchRows = size_t(1) << 20;
+static __device__ __align__(256) float g_builtin_scratch[kBuiltinScratchRows];
+
+// In host code `g_builtin_scratch` is only a handle for the runtime, not an address a kernel may
+// use; the device address is looked up once per device, with that device current.
+float* g_builtin_scratch_ptr[kMaxDevices] = {};
+
+int builtin_scratch(float** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return S2A_ERR_UNSUPPORTED;
+    if (!g_builtin_scratch_ptr[dev]) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_builtin_scratch);
+        if (e != cudaSuccess) return cuda_fail(e);
+        g_builtin_scratch_ptr[dev] = static_cast<float*>(ptr);
+    }
+    *out = g_builtin_scratch_ptr[dev];
+    return S2A_OK;
+}
+
+}  // namespace
+
+int s2a_bwd_noalloc(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO,
+                    void* dq, void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, void* stream) {
+    if (B <= 0 || N <= 0 || H <= 0) return S2A_ERR_INVALID_ARG;
+    if (static_cast<unsigned long long>(B) * static_cast<unsigned long long>(H) * static_cast<unsigned long long>(N) >
+        kBuiltinScratchRows)
+        return S2A_ERR_TOO_LARGE;
+    if (d <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
+    if (G % (2 * kTile) != 0) return (G > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
+    float* scratch = nullptr;
+    const int rc = builtin_scratch(&scratch);
+    if (rc != S2A_OK) return rc;
+    // Every row of D that the two gradient kernels read is rewritten by the first kernel of this
+    // call, so nothing left in the array by an earlier call has to be cleared.
+    return bwd_impl(q, k, v, o, lse, dO, dq, dk, dv, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2,
+                    G / 2, scratch, kBuiltinScratchRows * sizeof(float), stream, kStageAll);
+}
+
+size_t s2a_bwd_noalloc_max_rows(void) { return kBuiltinScratchRows; }
 
 int s2a_device_status(int* where) {
     DeviceState* ds = nullptr;

@@ -14,9 +14,9 @@
 // The roll of the shifted heads and the group boundaries are folded into TMA coordinates exactly
 // as in the forward kernel; all results are stored at original token rows.
 //
-// Both tensor-core kernels share one software pipeline (192 threads, one CTA per SM): warp 0
-// loads with TMA, warp 1 issues tcgen05 MMAs, warps 2-5 do the elementwise work with one
-// tensor-memory lane per thread.  The two score products of step n+1 are issued before the
+// Both tensor-core kernels share one software pipeline (320 threads, one CTA per SM): warp 0
+// loads with TMA, warp 1 issues tcgen05 MMAs, warps 2-9 do the elementwise work with one
+// tensor-memory lane and half of the columns per thread.  The two score products of step n+1 are issued before the
 // gradient products of step n, into the other half of a double buffer, so the elementwise work
 // of step n overlaps tensor-core work.
 #include "s2a_params.h"
@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(256) s2a_bwd_preprocess_kernel(const PreParams
 // ------------------------------------------------------------------------------------------------
 template <int HD>
 struct BwdCfg {
-    static constexpr int kThreads = 192;
+    static constexpr int kThreads = 320;  // TMA warp, MMA warp, 8 elementwise warps
     static constexpr int kBoxes = HD / 64;
     static constexpr int kBigBoxBytes = kTile * 128;            // 128-row box
     static constexpr int kSubBoxBytes = kSubTile * 128;         // 64-row box
@@ -95,11 +95,12 @@ __device__ __forceinline__ void pack32(const float (&x)[32], uint32_t (&out)[16]
     for (int e = 0; e < 16; ++e) out[e] = pack_bf16(x[2 * e], x[2 * e + 1]);
 }
 
-// Store one accumulator row (HD fp32 columns in tensor memory, times `mul`) as bf16.
-template <int HD>
-__device__ __forceinline__ void store_acc_row(uint32_t t_addr, float mul, __nv_bfloat16* dst_row) {
+// Store COLS consecutive fp32 accumulator columns of this thread's tensor-memory lane (times `mul`)
+// as bf16 to `dst`.
+template <int COLS>
+__device__ __forceinline__ void store_acc_cols(uint32_t t_addr, float mul, __nv_bfloat16* dst_row) {
 #pragma unroll
-    for (int c = 0; c < HD / 32; ++c) {
+    for (int c = 0; c < COLS / 32; ++c) {
         uint32_t r[32];
         tmem_ld_32x32(t_addr + c * 32, r);
         tmem_wait_ld();
@@ -115,6 +116,12 @@ __device__ __forceinline__ void store_acc_row(uint32_t t_addr, float mul, __nv_b
         }
     }
 }
+
+// The elementwise warps come in two groups of four: group `half` handles columns [32*half, +32) of
+// each 64-column score buffer and writes its 32 bf16 results (16 packed columns) over the start of
+// its own columns, so the two groups never touch each other's columns.  The 64 K values of the
+// bf16 operand therefore sit at packed columns [0,16) and [32,48) of the buffer:
+__device__ __forceinline__ uint32_t packed_operand_col(int kk) { return (kk >> 1) * 32 + (kk & 1) * 8; }
 
 // Barrier block common to both kernels.
 template <int kStages>
@@ -173,7 +180,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         mbar_init(&bars->drain, 1);
         for (int x = 0; x < 2; ++x) {
             mbar_init(&bars->s_full[x], 1);
-            mbar_init(&bars->p_full[x], 128);
+            mbar_init(&bars->p_full[x], 256);
         }
         for (int st = 0; st < C::kStages; ++st) {
             mbar_init(&bars->st_full[st], 1);
@@ -229,28 +236,24 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         if (lane == 0) {
             constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);  // S = Q K^T, dP = dO V^T
             constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);       // dQ += dS K   (K is MN-major)
-            const uint32_t aQ = smem_u32(sQ), aDO = smem_u32(sDO);
+            const uint32_t dQ = desc_lo_k_major(smem_u32(sQ)), dDO = desc_lo_k_major(smem_u32(sDO));
             // score products of step n into buffer n & 1
             auto issue_scores = [&](int n) -> bool {
                 const int st = n % C::kStages;
                 if (!mbar_wait(&bars->st_full[st], (n / C::kStages) & 1, ctx, kWaitBwdDq + 2)) return false;
                 tc_fence_after();
                 const uint32_t aK = smem_u32(sStage + st * C::kStageBytes);
-                const uint32_t aV = aK + C::kSubTileBytes;
+                const uint32_t dK = desc_lo_k_major(aK), dV = desc_lo_k_major(aK + C::kSubTileBytes);
                 const uint32_t tS = tmem_base + kColS + (n & 1) * kSubTile;
                 const uint32_t tP = tmem_base + kColP + (n & 1) * kSubTile;
 #pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t offA = (kk >> 2) * C::kBigBoxBytes + (kk & 3) * 32;
-                    const uint32_t offB = (kk >> 2) * C::kSubBoxBytes + (kk & 3) * 32;
-                    mma_ss(tS, desc_k_major(aQ + offA), desc_k_major(aK + offB), idesc_sc, kk > 0);
-                }
+                for (int kk = 0; kk < HD / 16; ++kk)
+                    mma_ss(tS, dQ + desc_step_k_major(kk, C::kBigBoxBytes), dK + desc_step_k_major(kk, C::kSubBoxBytes),
+                           idesc_sc, kk > 0);
 #pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t offA = (kk >> 2) * C::kBigBoxBytes + (kk & 3) * 32;
-                    const uint32_t offB = (kk >> 2) * C::kSubBoxBytes + (kk & 3) * 32;
-                    mma_ss(tP, desc_k_major(aDO + offA), desc_k_major(aV + offB), idesc_sc, kk > 0);
-                }
+                for (int kk = 0; kk < HD / 16; ++kk)
+                    mma_ss(tP, dDO + desc_step_k_major(kk, C::kBigBoxBytes), dV + desc_step_k_major(kk, C::kSubBoxBytes),
+                           idesc_sc, kk > 0);
                 mma_commit(&bars->s_full[n & 1]);
                 return true;
             };
@@ -261,12 +264,12 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
                 if (!mbar_wait(&bars->p_full[n & 1], (n >> 1) & 1, ctx, kWaitBwdDq + 4)) break;
                 tc_fence_after();
                 const int st = n % C::kStages;
-                const uint32_t aK = smem_u32(sStage + st * C::kStageBytes);
+                const uint32_t dKmn = desc_lo_mn_major(smem_u32(sStage + st * C::kStageBytes), C::kSubBoxBytes);
                 const uint32_t tdS = tmem_base + kColS + (n & 1) * kSubTile;  // bf16 dS over the S buffer
 #pragma unroll
                 for (int kk = 0; kk < kSubTile / 16; ++kk)
-                    mma_ts(tmem_base + kColAcc, tdS + kk * 8, desc_mn_major(aK + kk * 2048, C::kSubBoxBytes),
-                           idesc_acc, (n > 0) || (kk > 0));
+                    mma_ts(tmem_base + kColAcc, tdS + packed_operand_col(kk), dKmn + kk * kDescStepMn, idesc_acc,
+                           (n > 0) || (kk > 0));
                 mma_commit(&bars->st_empty[st]);
                 if (n == n_steps - 1) mma_commit(&bars->acc_full);
             }
@@ -278,6 +281,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         __syncwarp();
     } else {
         const int quad = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int row = quad * 32 + lane;
         const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
         const size_t stat_idx = (static_cast<size_t>(b) * geo.H + h) * geo.N + tq0 + row;
@@ -288,27 +292,32 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         for (int n = 0; n < n_steps; ++n) {
             if (!mbar_wait(&bars->s_full[n & 1], (n >> 1) & 1, ctx, kWaitBwdDq + 5)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t tS = t_row + kColS + (n & 1) * kSubTile;
-            const uint32_t tP = t_row + kColP + (n & 1) * kSubTile;
-            // key x of this sub-tile is visible to query row r iff 64 n + x <= 128 i + r
-            const int lim = i * kTile + row - n * kSubTile;  // visible iff x <= lim
-#pragma unroll
-            for (int c = 0; c < kSubTile / 32; ++c) {
-                uint32_t sr[32], pr[32];
-                tmem_ld_32x32(tS + c * 32, sr);
-                tmem_ld_32x32(tP + c * 32, pr);
-                tmem_wait_ld();
-                float ds[32];
+            const uint32_t tS = t_row + kColS + (n & 1) * kSubTile + half * 32;
+            const uint32_t tP = t_row + kColP + (n & 1) * kSubTile + half * 32;
+            uint32_t sr[32], pr[32];
+            tmem_ld_32x32(tS, sr);
+            tmem_ld_32x32(tP, pr);
+            tmem_wait_ld();
+            float ds[32];
+            if (n >= 2 * i) {
+                // diagonal sub-tiles: key x is visible to query row r iff 64 n + x <= 128 i + r
+                const int lim = i * kTile + row - n * kSubTile - half * 32;  // visible iff e <= lim
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
                     float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, neg_lse2));
-                    if (c * 32 + e > lim) pe = 0.f;
+                    if (e > lim) pe = 0.f;
                     ds[e] = pe * (__uint_as_float(pr[e]) - Drow);
                 }
-                uint32_t pk[16];
-                pack32(ds, pk);
-                tmem_st_32x16(tS + c * 16, pk);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, neg_lse2));
+                    ds[e] = pe * (__uint_as_float(pr[e]) - Drow);
+                }
             }
+            uint32_t pk[16];
+            pack32(ds, pk);
+            tmem_st_32x16(tS, pk);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(&bars->p_full[n & 1]);
@@ -316,7 +325,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDq + 6)) {
             tc_fence_after();
             __nv_bfloat16* dst = p.dq + ((static_cast<size_t>(b) * geo.N + tq0 + row) * geo.H + h) * HD;
-            store_acc_row<HD>(t_row + kColAcc, p.scale, dst);
+            store_acc_cols<HD / 2>(t_row + kColAcc + half * (HD / 2), p.scale, dst + half * (HD / 2));
         }
     }
 
@@ -399,7 +408,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         mbar_init(&bars->drain, 1);
         for (int x = 0; x < 2; ++x) {
             mbar_init(&bars->s_full[x], 1);
-            mbar_init(&bars->p_full[x], 128);
+            mbar_init(&bars->p_full[x], 256);
         }
         for (int st = 0; st < C::kStages; ++st) {
             mbar_init(&bars->st_full[st], 1);
@@ -463,27 +472,23 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         if (lane == 0) {
             constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);  // S^T = K Q^T, dP^T = V dO^T
             constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);       // dV += P^T dO, dK += dS^T Q
-            const uint32_t aK = smem_u32(sK), aV = smem_u32(sV);
+            const uint32_t dK = desc_lo_k_major(smem_u32(sK)), dV = desc_lo_k_major(smem_u32(sV));
             auto issue_scores = [&](int it) -> bool {
                 const int st = it % C::kStages;
                 if (!mbar_wait(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 2)) return false;
                 tc_fence_after();
                 const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
-                const uint32_t aDO = aQ + C::kSubTileBytes;
+                const uint32_t dQ = desc_lo_k_major(aQ), dDO = desc_lo_k_major(aQ + C::kSubTileBytes);
                 const uint32_t tS = tmem_base + kColS + (it & 1) * kSubTile;
                 const uint32_t tP = tmem_base + kColP + (it & 1) * kSubTile;
 #pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t offA = (kk >> 2) * C::kBigBoxBytes + (kk & 3) * 32;
-                    const uint32_t offB = (kk >> 2) * C::kSubBoxBytes + (kk & 3) * 32;
-                    mma_ss(tS, desc_k_major(aK + offA), desc_k_major(aQ + offB), idesc_sc, kk > 0);
-                }
+                for (int kk = 0; kk < HD / 16; ++kk)
+                    mma_ss(tS, dK + desc_step_k_major(kk, C::kBigBoxBytes), dQ + desc_step_k_major(kk, C::kSubBoxBytes),
+                           idesc_sc, kk > 0);
 #pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t offA = (kk >> 2) * C::kBigBoxBytes + (kk & 3) * 32;
-                    const uint32_t offB = (kk >> 2) * C::kSubBoxBytes + (kk & 3) * 32;
-                    mma_ss(tP, desc_k_major(aV + offA), desc_k_major(aDO + offB), idesc_sc, kk > 0);
-                }
+                for (int kk = 0; kk < HD / 16; ++kk)
+                    mma_ss(tP, dV + desc_step_k_major(kk, C::kBigBoxBytes), dDO + desc_step_k_major(kk, C::kSubBoxBytes),
+                           idesc_sc, kk > 0);
                 mma_commit(&bars->s_full[it & 1]);
                 return true;
             };
@@ -495,17 +500,18 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                 tc_fence_after();
                 const int st = it % C::kStages;
                 const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
-                const uint32_t aDO = aQ + C::kSubTileBytes;
+                const uint32_t dQmn = desc_lo_mn_major(aQ, C::kSubBoxBytes);
+                const uint32_t dDOmn = desc_lo_mn_major(aQ + C::kSubTileBytes, C::kSubBoxBytes);
                 const uint32_t tPt = tmem_base + kColS + (it & 1) * kSubTile;   // bf16 P^T over the S^T buffer
                 const uint32_t tdSt = tmem_base + kColP + (it & 1) * kSubTile;  // bf16 dS^T over the dP^T buffer
 #pragma unroll
                 for (int kk = 0; kk < kSubTile / 16; ++kk)
-                    mma_ts(tmem_base + kColDV, tPt + kk * 8, desc_mn_major(aDO + kk * 2048, C::kSubBoxBytes),
-                           idesc_acc, (it > 0) || (kk > 0));
+                    mma_ts(tmem_base + kColDV, tPt + packed_operand_col(kk), dDOmn + kk * kDescStepMn, idesc_acc,
+                           (it > 0) || (kk > 0));
 #pragma unroll
                 for (int kk = 0; kk < kSubTile / 16; ++kk)
-                    mma_ts(tmem_base + kColDK, tdSt + kk * 8, desc_mn_major(aQ + kk * 2048, C::kSubBoxBytes),
-                           idesc_acc, (it > 0) || (kk > 0));
+                    mma_ts(tmem_base + kColDK, tdSt + packed_operand_col(kk), dQmn + kk * kDescStepMn, idesc_acc,
+                           (it > 0) || (kk > 0));
                 mma_commit(&bars->st_empty[st]);
                 if (it == total_steps - 1) mma_commit(&bars->acc_full);
             }
@@ -517,6 +523,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         __syncwarp();
     } else {
         const int quad = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int row = quad * 32 + lane;  // key row of the tile owned by this thread
         const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
         const float c2 = p.scale_log2;
@@ -530,40 +537,38 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                 if (!mbar_wait(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 5)) { ok = false; break; }
                 if (!mbar_wait(&bars->s_full[it & 1], (it >> 1) & 1, ctx, kWaitBwdDkDv + 6)) { ok = false; break; }
                 tc_fence_after();
-                const float4* lse4 = reinterpret_cast<const float4*>(sStat + st * 2 * kSubTile);
+                const float4* lse4 = reinterpret_cast<const float4*>(sStat + st * 2 * kSubTile) + half * 8;
                 const float4* d4 = lse4 + kSubTile / 4;
-                const uint32_t tS = t_row + kColS + (it & 1) * kSubTile;
-                const uint32_t tP = t_row + kColP + (it & 1) * kSubTile;
+                const uint32_t tS = t_row + kColS + (it & 1) * kSubTile + half * 32;
+                const uint32_t tP = t_row + kColP + (it & 1) * kSubTile + half * 32;
+                uint32_t sr[32], pr[32];
+                tmem_ld_32x32(tS, sr);
+                tmem_ld_32x32(tP, pr);
+                tmem_wait_ld();
+                float pt[32], ds[32];
                 // query x of this sub-tile sees key row r iff 128 j + r <= 64 n + x
-                const int lim = w.j * kTile + row - n * kSubTile;  // visible iff x >= lim
+                const bool diagonal = n < w.n_begin + 2;
+                const int lim = diagonal ? w.j * kTile + row - n * kSubTile - half * 32 : -1;  // visible iff e >= lim
 #pragma unroll
-                for (int c = 0; c < kSubTile / 32; ++c) {
-                    uint32_t sr[32], pr[32];
-                    tmem_ld_32x32(tS + c * 32, sr);
-                    tmem_ld_32x32(tP + c * 32, pr);
-                    tmem_wait_ld();
-                    float pt[32], ds[32];
+                for (int e4 = 0; e4 < 8; ++e4) {
+                    const float4 l = lse4[e4];
+                    const float4 dd = d4[e4];
+                    const float lv[4] = {l.x, l.y, l.z, l.w};
+                    const float dv[4] = {dd.x, dd.y, dd.z, dd.w};
 #pragma unroll
-                    for (int e4 = 0; e4 < 8; ++e4) {
-                        const float4 l = lse4[c * 8 + e4];
-                        const float4 dd = d4[c * 8 + e4];
-                        const float lv[4] = {l.x, l.y, l.z, l.w};
-                        const float dv[4] = {dd.x, dd.y, dd.z, dd.w};
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int e = e4 * 4 + u;
-                            float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, -lv[u] * kLog2e));
-                            if (c * 32 + e < lim) pe = 0.f;
-                            pt[e] = pe;
-                            ds[e] = pe * (__uint_as_float(pr[e]) - dv[u]);
-                        }
+                    for (int u = 0; u < 4; ++u) {
+                        const int e = e4 * 4 + u;
+                        float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, -lv[u] * kLog2e));
+                        if (diagonal && e < lim) pe = 0.f;
+                        pt[e] = pe;
+                        ds[e] = pe * (__uint_as_float(pr[e]) - dv[u]);
                     }
-                    uint32_t pk[16];
-                    pack32(pt, pk);
-                    tmem_st_32x16(tS + c * 16, pk);
-                    pack32(ds, pk);
-                    tmem_st_32x16(tP + c * 16, pk);
                 }
+                uint32_t pk[16];
+                pack32(pt, pk);
+                tmem_st_32x16(tS, pk);
+                pack32(ds, pk);
+                tmem_st_32x16(tP, pk);
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(&bars->p_full[it & 1]);
@@ -572,8 +577,8 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDkDv + 7)) {
             tc_fence_after();
             const size_t out_row = ((static_cast<size_t>(b) * geo.N + tk0 + row) * geo.Hkv + hk) * HD;
-            store_acc_row<HD>(t_row + kColDV, 1.0f, p.dv + out_row);
-            store_acc_row<HD>(t_row + kColDK, p.scale, p.dk + out_row);
+            if (half == 0) store_acc_cols<HD>(t_row + kColDV, 1.0f, p.dv + out_row);
+            else store_acc_cols<HD>(t_row + kColDK, p.scale, p.dk + out_row);
         }
     }
 

@@ -8,9 +8,10 @@
 // positions -- for the wrapped last group of a shifted head that is the range [N-G/2, N) followed
 // by [0, G/2).  Outputs are stored at the original token rows, which is the roll back.
 //
-// Warp roles (192 threads): warp 0 issues TMA loads, warp 1 owns tensor memory and issues the
-// tcgen05 MMAs, warps 2-5 hold one score row per thread (tcgen05.ld 32x32b) and run the online
-// softmax.  S = Q K^T accumulates in tensor memory, P (bf16) is written back over S and used as the
+// Warp roles (320 threads): warp 0 issues TMA loads, warp 1 owns tensor memory and issues the
+// tcgen05 MMAs, warps 2-9 run the online softmax: a score row lives in one tensor-memory lane
+// (tcgen05.ld 32x32b) and is shared by two threads, one per 64-column half, which exchange their
+// partial row maxima through shared memory.  S = Q K^T accumulates in tensor memory, P (bf16) is written back over S and used as the
 // tensor-memory A operand of O += P V; O stays in tensor memory until the epilogue.  Two CTAs fit
 // on one SM, so one CTA's softmax overlaps the other CTA's MMAs.
 #include "s2a_params.h"
@@ -22,12 +23,12 @@ namespace {
 
 template <int HD>
 struct FwdCfg {
-    static constexpr int kThreads = 192;
+    static constexpr int kThreads = 320;
     static constexpr int kBoxes = HD / 64;                      // 64-column TMA boxes per tile
     static constexpr int kBoxBytes = kTile * 128;               // 128 rows x 128 bytes
     static constexpr int kTileBytes = kBoxes * kBoxBytes;       // one Q, K or V tile
     static constexpr int kStages = (HD == 128) ? 1 : 2;         // K/V ring depth
-    static constexpr int kBarBytes = 256;
+    static constexpr int kBarBytes = 256 + 2 * 2 * 128 * 8;  // barriers + row-max exchange slots
     static constexpr int kSmemBytes = 1024 /* alignment slack */ + (1 + 2 * kStages) * kTileBytes + kBarBytes;
     static constexpr int kTmemCols = 256;                       // S: [0,128)  O: [128, 128+HD)
     static constexpr int kColS = 0;
@@ -58,6 +59,8 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
     uint64_t* v_empty = v_full + C::kStages;     // [kStages]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(v_empty + C::kStages);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    // exchange slots between the two threads of a row: [2 parities][2 halves][128 rows] x {value, sequence}
+    volatile float2* xch = reinterpret_cast<volatile float2*>(reinterpret_cast<uint8_t*>(bars) + 256);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -90,7 +93,7 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
         mbar_init(s_full, 1);
-        mbar_init(p_full, 128);
+        mbar_init(p_full, 256);
         mbar_init(o_full, 1);
         mbar_init(drain, 1);
         for (int st = 0; st < C::kStages; ++st) {
@@ -104,6 +107,9 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
         tma_prefetch_desc(&p.tm_q);
         tma_prefetch_desc(&p.tm_k);
         tma_prefetch_desc(&p.tm_v);
+    }
+    for (int idx = threadIdx.x; idx < 2 * 2 * 128; idx += C::kThreads) {  // sequence 0 = "nothing published"
+        const_cast<float2*>(xch)[idx] = make_float2(0.f, 0.f);
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, C::kTmemCols);
@@ -152,21 +158,21 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
             constexpr uint32_t idesc_o = idesc_bf16(128, HD, 0, 1);   // O += P V    (V is MN-major)
             const uint32_t tS = tmem_base + C::kColS;
             const uint32_t tO = tmem_base + C::kColO;
-            const uint32_t aQ = smem_u32(sQ);
+            const uint32_t dQ = desc_lo_k_major(smem_u32(sQ));
             bool ok = mbar_wait(q_full, 0, ctx, kWaitFwd + 3);
             for (int j = 0; ok && j < n_kv; ++j) {
                 const int st = j % C::kStages;
                 const uint32_t ph = (j / C::kStages) & 1;
-                const uint32_t aK = smem_u32(sK + st * C::kTileBytes);
-                const uint32_t aV = smem_u32(sV + st * C::kTileBytes);
+                const uint32_t dK = desc_lo_k_major(smem_u32(sK + st * C::kTileBytes));
+                const uint32_t dV = desc_lo_mn_major(smem_u32(sV + st * C::kTileBytes), C::kBoxBytes);
                 if (!mbar_wait(k_full + st, ph, ctx, kWaitFwd + 4)) break;
                 tc_fence_after();
                 // The previous P (aliased on S) was consumed by the previous P.V, which precedes
                 // this MMA in issue order; the softmax warps finished reading S before that.
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * C::kBoxBytes + (kk & 3) * 32;
-                    mma_ss(tS, desc_k_major(aQ + off), desc_k_major(aK + off), idesc_s, kk > 0);
+                    constexpr uint32_t kBox = C::kBoxBytes;
+                    mma_ss(tS, dQ + desc_step_k_major(kk, kBox), dK + desc_step_k_major(kk, kBox), idesc_s, kk > 0);
                 }
                 mma_commit(k_empty + st);
                 mma_commit(s_full);
@@ -175,7 +181,7 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < kTile / 16; ++kk) {
-                    mma_ts(tO, tS + kk * 8, desc_mn_major(aV + kk * 2048, C::kBoxBytes), idesc_o, (j > 0) || (kk > 0));
+                    mma_ts(tO, tS + (kk >> 2) * 64 + (kk & 3) * 8, dV + kk * kDescStepMn, idesc_o, (j > 0) || (kk > 0));
                 }
                 mma_commit(v_empty + st);
                 if (j == n_kv - 1) mma_commit(o_full);
@@ -189,81 +195,136 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
         __syncwarp();
     } else {
         // =========================== softmax + epilogue ======================================
+        // Thread (quad, lane, half) owns columns [64*half, +64) of score row 32*quad + lane.  Its
+        // bf16 P values go over the first 32 of its own columns, so the two halves never write
+        // into columns the other half still has to read: P's 128 K values sit at packed columns
+        // [0,32) and [64,96).
         const int quad = warp & 3;             // tensor-memory lane quadrant this warp may access
-        const int row = quad * 32 + lane;      // row of the query tile owned by this thread
+        const int half = (warp - 2) >> 2;
+        const int row = quad * 32 + lane;
         const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+        const uint32_t t_mine = t_row + C::kColS + half * 64;
         const float c2 = p.scale_log2;
-        float m_used = -INFINITY;              // running maximum, already scaled to log2 units
-        float l = 0.f;                         // running sum of exp2(s*c2 - m_used)
+        float m_used = -INFINITY;              // running maximum in use, already scaled to log2 units
+        float l = 0.f;                         // this half's part of the running sum of exp2(s*c2 - m_used)
         bool ok = true;
+        // Publish `v` to the thread that owns the other half of this row and fetch its value.
+        // One 8-byte store carries the value together with a sequence number, the reader polls
+        // (bounded) until the number matches.  Slots alternate with the parity of `seq`; a thread
+        // cannot run two exchanges ahead of its partner, so a slot is never overwritten unread.
+        auto pair_exchange = [&](float v, int seq, float& other) -> bool {
+            const uint32_t slot = smem_u32(const_cast<float2*>(xch)) + (seq & 1) * 2048;
+            const uint32_t mine = slot + (half * 128 + row) * 8;
+            const uint32_t theirs = slot + ((half ^ 1) * 128 + row) * 8;
+            asm volatile("st.volatile.shared.v2.b32 [%0], {%1, %2};" ::"r"(mine), "r"(__float_as_uint(v)), "r"(seq + 1)
+                         : "memory");
+            const long long t0 = clock64();
+            for (uint32_t spins = 1;; ++spins) {
+                uint32_t val, tag;
+                asm volatile("ld.volatile.shared.v2.b32 {%0, %1}, [%2];" : "=r"(val), "=r"(tag) : "r"(theirs) : "memory");
+                if (tag == static_cast<uint32_t>(seq + 1)) {
+                    other = __uint_as_float(val);
+                    return true;
+                }
+                if ((spins & 255u) == 0) {
+                    if (*abort_flag != 0) return false;
+                    if (clock64() - t0 > kWaitLimitCycles) {
+                        *abort_flag = kWaitFwd + 9;
+                        atomicCAS(p.status, 0, kWaitFwd + 9);
+                        return false;
+                    }
+                }
+            }
+        };
         for (int j = 0; j < n_kv; ++j) {
             if (!mbar_wait(s_full, j & 1, ctx, kWaitFwd + 7)) { ok = false; break; }
             tc_fence_after();
-            uint32_t sreg[4][32];
+            // pass 1: row maximum of this thread's 64 columns (the scores are read again in pass 2,
+            // 32 at a time, which keeps the register footprint small enough for two CTAs per SM)
+            const bool diagonal = (j == i);    // key x of the tile is visible to query row r iff x <= r
+            const int lim = row - half * 64;   // visible iff (column within this half) <= lim
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld_32x32(t_row + C::kColS + c * 32, sreg[c]);
-            tmem_wait_ld();
-            if (j == i) {
-                // diagonal tile: key x of the tile is visible to query row r iff x <= r
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
+            for (int c = 0; c < 2; ++c) {
+                uint32_t sreg[32];
+                tmem_ld_32x32(t_mine + c * 32, sreg);
+                tmem_wait_ld();
+                if (diagonal) {
 #pragma unroll
                     for (int e = 0; e < 32; ++e)
-                        if (c * 32 + e > row) sreg[c][e] = 0xff800000u;  // -inf
+                        if (c * 32 + e > lim) sreg[e] = 0xff800000u;  // -inf
+                }
+#pragma unroll
+                for (int e = 0; e < 32; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], __uint_as_float(sreg[e]));
             }
-            float mx = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-#pragma unroll
-                for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(sreg[c][e]));
+            const float mx_own = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            float mx_other;
+            if (!pair_exchange(mx_own, j, mx_other)) { ok = false; break; }
+            const float mx = fmaxf(mx_own, mx_other);
             const float m_new = fmaxf(m_used, mx * c2);
             if (j == 0) {
                 m_used = m_new;
             } else {
                 const bool need = (m_new - m_used) > kLazyRescale;
                 if (__any_sync(0xffffffffu, need)) {
-                    // s_full(j) also covers the previous P.V, so O is quiescent here
+                    // s_full(j) also covers the previous P.V, so O is quiescent here; each half
+                    // rescales its own half of O's columns
                     const float alpha = need ? fast_exp2(m_used - m_new) : 1.0f;
                     l *= alpha;
 #pragma unroll
-                    for (int c = 0; c < HD / 32; ++c) {
+                    for (int c = 0; c < HD / 64; ++c) {
                         uint32_t oreg[32];
-                        tmem_ld_32x32(t_row + C::kColO + c * 32, oreg);
+                        const uint32_t t_o = t_row + C::kColO + half * (HD / 2) + c * 32;
+                        tmem_ld_32x32(t_o, oreg);
                         tmem_wait_ld();
 #pragma unroll
                         for (int e = 0; e < 32; ++e) oreg[e] = __float_as_uint(__uint_as_float(oreg[e]) * alpha);
-                        tmem_st_32x32(t_row + C::kColO + c * 32, oreg);
+                        tmem_st_32x32(t_o, oreg);
                     }
                     if (need) m_used = m_new;
                 }
             }
-            float sum = 0.f;
+            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
+                uint32_t sreg[32];
+                tmem_ld_32x32(t_mine + c * 32, sreg);
+                tmem_wait_ld();
+                if (diagonal) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (c * 32 + e > lim) sreg[e] = 0xff800000u;
+                }
                 uint32_t preg[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
-                    const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[c][2 * e]), c2, -m_used));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[c][2 * e + 1]), c2, -m_used));
-                    sum += p0 + p1;
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[2 * e]), c2, -m_used));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[2 * e + 1]), c2, -m_used));
+                    sum4[e & 3] += p0 + p1;
                     preg[e] = pack_bf16(p0, p1);
                 }
-                tmem_st_32x16(t_row + C::kColS + c * 16, preg);
+                // packed columns [16c, 16c+16) overlay score columns [16c, 16c+16) of this half, which
+                // pass 2 has already consumed (c = 1 writes over columns 16..31, read when c was 0)
+                tmem_st_32x16(t_mine + c * 16, preg);
             }
-            l += sum;
+            l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(p_full);
         }
         if (ok && mbar_wait(o_full, 0, ctx, kWaitFwd + 8)) {
             tc_fence_after();
-            const float inv_l = 1.0f / l;
+            // total row sum = this half's part + the other half's
+            float l_other = 0.f;
+            pair_exchange(l, n_kv, l_other);
+            const float l_row = l + l_other;
+            const float inv_l = 1.0f / l_row;
             const int t = tq0 + row;
-            __nv_bfloat16* orow = p.o + ((static_cast<size_t>(b) * p.geo.N + t) * p.geo.H + h) * HD;
+            __nv_bfloat16* orow = p.o + ((static_cast<size_t>(b) * p.geo.N + t) * p.geo.H + h) * HD + half * (HD / 2);
 #pragma unroll
-            for (int c = 0; c < HD / 32; ++c) {
+            for (int c = 0; c < HD / 64; ++c) {
                 uint32_t oreg[32];
-                tmem_ld_32x32(t_row + C::kColO + c * 32, oreg);
+                tmem_ld_32x32(t_row + C::kColO + half * (HD / 2) + c * 32, oreg);
                 tmem_wait_ld();
                 uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
 #pragma unroll
@@ -277,7 +338,8 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
                 }
             }
             // natural-log sum-exp of the scaled scores
-            p.lse[(static_cast<size_t>(b) * p.geo.H + h) * p.geo.N + t] = (m_used + log2f(l)) * 0.6931471805599453f;
+            if (half == 0)
+                p.lse[(static_cast<size_t>(b) * p.geo.H + h) * p.geo.N + t] = (m_used + log2f(l_row)) * 0.6931471805599453f;
         }
     }
 

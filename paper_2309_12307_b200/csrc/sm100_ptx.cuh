@@ -184,23 +184,31 @@ __device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint32_t (&r
 // leaves behind: row r at byte r * 128, its 16-byte chunks permuted by (r & 7); 8 rows = one
 // 1024-byte swizzle atom.  The tile base must be 1024-byte aligned.
 
-constexpr uint64_t kDescVersion = 1ull << 46;   // descriptor version field for this architecture
-constexpr uint64_t kDescSwizzle128 = 2ull << 61;
 constexpr uint32_t kSwizzleAtomBytes = 1024;
+// A 64-bit shared-memory descriptor is {low word, high word}.  The high word is the same for every
+// operand used here: stride between 8-row groups (1024 B >> 4) in bits 0-13, descriptor version 1
+// in bit 14 (bit 46 of the descriptor), 128-byte swizzle (code 2) in bits 29-31 (bits 61-63).
+// The low word carries the start address (>> 4, bits 0-13) and the leading-dimension offset
+// (>> 4, bits 16-29), so stepping through a tile is a 32-bit add on the low word: the MMA-issuing
+// thread is a single instruction stream and every instruction it spends on address arithmetic
+// delays the tensor pipe.
+constexpr uint32_t kDescHi = (kSwizzleAtomBytes >> 4) | (1u << 14) | (2u << 29);
 
 // Operand whose contraction (K) index runs along the 128-byte rows ("K-major"): rows are the M or N
-// index.  `saddr` may point 32 * kk bytes into the first row to select the kk-th group of 16 K values.
-__device__ __forceinline__ uint64_t desc_k_major(uint32_t saddr) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) /* leading offset: unused here */ |
-           ((uint64_t)(kSwizzleAtomBytes >> 4) << 32) /* 8-row group stride */ | kDescVersion | kDescSwizzle128;
+// index.  Add desc_step_k_major(kk, box_bytes) to reach the kk-th group of 16 K values.
+__device__ __forceinline__ uint32_t desc_lo_k_major(uint32_t saddr) {
+    return ((saddr & 0x3FFFFu) >> 4) | (1u << 16);  // leading offset unused for this layout
+}
+__host__ __device__ constexpr uint32_t desc_step_k_major(int kk, uint32_t box_bytes) {
+    return ((kk >> 2) * box_bytes + (kk & 3) * 32u) >> 4;  // 4 groups of 16 per 64-column box
 }
 // Operand whose M or N index runs along the 128-byte rows ("MN-major"): rows are the K index.
 // `block_stride_bytes` is the distance between consecutive 64-wide blocks of the M/N index (the
-// size of one TMA box); groups of 8 K rows are 1024 bytes apart.  Advance K by 16: saddr += 2048.
-__device__ __forceinline__ uint64_t desc_mn_major(uint32_t saddr, uint32_t block_stride_bytes) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)((block_stride_bytes >> 4) & 0x3FFFu) << 16) |
-           ((uint64_t)(kSwizzleAtomBytes >> 4) << 32) | kDescVersion | kDescSwizzle128;
+// size of one TMA box); groups of 8 K rows are 1024 bytes apart.  16 K rows further: + kDescStepMn.
+__device__ __forceinline__ uint32_t desc_lo_mn_major(uint32_t saddr, uint32_t block_stride_bytes) {
+    return ((saddr & 0x3FFFFu) >> 4) | (((block_stride_bytes >> 4) & 0x3FFFu) << 16);
 }
+constexpr uint32_t kDescStepMn = 2048u >> 4;
 
 // Instruction descriptor for kind::f16 with bf16 A and B, fp32 D, M x N tile.
 // a_mn / b_mn: operand is MN-major (1) or K-major (0).
@@ -214,28 +222,33 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N, int a_mn, int b_
            | ((uint32_t)(M >> 4) << 24);  // M / 16
 }
 
-// D[tmem] (+)= A[smem] * B[smem]; issued by ONE thread.
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+// D[tmem] (+)= A[smem] * B[smem]; issued by ONE thread.  a_lo / b_lo: descriptor low words.
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
                                        uint32_t accumulate) {
     asm volatile(
         "{\n"
         ".reg .pred p;\n"
+        ".reg .b64 da, db;\n"
+        "mov.b64 da, {%1, %5};\n"
+        "mov.b64 db, {%2, %5};\n"
         "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n"
         "}\n" ::"r"(d_tmem),
-        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
         : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]; A holds bf16 pairs, one M row per lane, 16 K values per 8 columns.
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc,
                                        uint32_t accumulate) {
     asm volatile(
         "{\n"
         ".reg .pred p;\n"
+        ".reg .b64 db;\n"
+        "mov.b64 db, {%2, %5};\n"
         "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n"
         "}\n" ::"r"(d_tmem),
-        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
         : "memory");
 }
 // Arrive once on `bar` when every MMA this thread issued so far has completed.

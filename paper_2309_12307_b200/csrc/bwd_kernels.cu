@@ -233,19 +233,21 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);  // S = Q K^T, dP = dO V^T
-            constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);       // dQ += dS K   (K is MN-major)
-            const uint32_t dQ = desc_lo_k_major(smem_u32(sQ)), dDO = desc_lo_k_major(smem_u32(sDO));
-            // score products of step n into buffer n & 1
-            auto issue_scores = [&](int n) -> bool {
-                const int st = n % C::kStages;
-                if (!mbar_wait(&bars->st_full[st], (n / C::kStages) & 1, ctx, kWaitBwdDq + 2)) return false;
-                tc_fence_after();
-                const uint32_t aK = smem_u32(sStage + st * C::kStageBytes);
-                const uint32_t dK = desc_lo_k_major(aK), dV = desc_lo_k_major(aK + C::kSubTileBytes);
-                const uint32_t tS = tmem_base + kColS + (n & 1) * kSubTile;
-                const uint32_t tP = tmem_base + kColP + (n & 1) * kSubTile;
+        // The whole warp walks the loop so that addresses and descriptors stay warp-uniform values;
+        // only the MMA and commit instructions themselves are issued by one elected lane.
+        constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);  // S = Q K^T, dP = dO V^T
+        constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);       // dQ += dS K   (K is MN-major)
+        const uint32_t dQ = desc_lo_k_major(smem_u32(sQ)), dDO = desc_lo_k_major(smem_u32(sDO));
+        // score products of step n into buffer n & 1
+        auto issue_scores = [&](int n) -> bool {
+            const int st = n % C::kStages;
+            if (!mbar_wait_uniform(&bars->st_full[st], (n / C::kStages) & 1, ctx, kWaitBwdDq + 2)) return false;
+            tc_fence_after();
+            const uint32_t aK = smem_u32(sStage + st * C::kStageBytes);
+            const uint32_t dK = desc_lo_k_major(aK), dV = desc_lo_k_major(aK + C::kSubTileBytes);
+            const uint32_t tS = tmem_base + kColS + (n & 1) * kSubTile;
+            const uint32_t tP = tmem_base + kColP + (n & 1) * kSubTile;
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk)
                     mma_ss(tS, dQ + desc_step_k_major(kk, C::kBigBoxBytes), dK + desc_step_k_major(kk, C::kSubBoxBytes),
@@ -255,17 +257,20 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
                     mma_ss(tP, dDO + desc_step_k_major(kk, C::kBigBoxBytes), dV + desc_step_k_major(kk, C::kSubBoxBytes),
                            idesc_sc, kk > 0);
                 mma_commit(&bars->s_full[n & 1]);
-                return true;
-            };
-            bool ok = mbar_wait(&bars->res_full, 0, ctx, kWaitBwdDq + 3);
-            ok = ok && issue_scores(0);
-            for (int n = 0; ok && n < n_steps; ++n) {
-                if (n + 1 < n_steps && !issue_scores(n + 1)) break;
-                if (!mbar_wait(&bars->p_full[n & 1], (n >> 1) & 1, ctx, kWaitBwdDq + 4)) break;
-                tc_fence_after();
-                const int st = n % C::kStages;
-                const uint32_t dKmn = desc_lo_mn_major(smem_u32(sStage + st * C::kStageBytes), C::kSubBoxBytes);
-                const uint32_t tdS = tmem_base + kColS + (n & 1) * kSubTile;  // bf16 dS over the S buffer
+            }
+            __syncwarp();
+            return true;
+        };
+        bool ok = mbar_wait_uniform(&bars->res_full, 0, ctx, kWaitBwdDq + 3);
+        ok = ok && issue_scores(0);
+        for (int n = 0; ok && n < n_steps; ++n) {
+            if (n + 1 < n_steps && !issue_scores(n + 1)) break;
+            if (!mbar_wait_uniform(&bars->p_full[n & 1], (n >> 1) & 1, ctx, kWaitBwdDq + 4)) break;
+            tc_fence_after();
+            const int st = n % C::kStages;
+            const uint32_t dKmn = desc_lo_mn_major(smem_u32(sStage + st * C::kStageBytes), C::kSubBoxBytes);
+            const uint32_t tdS = tmem_base + kColS + (n & 1) * kSubTile;  // bf16 dS over the S buffer
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kSubTile / 16; ++kk)
                     mma_ts(tmem_base + kColAcc, tdS + packed_operand_col(kk), dKmn + kk * kDescStepMn, idesc_acc,
@@ -273,7 +278,10 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
                 mma_commit(&bars->st_empty[st]);
                 if (n == n_steps - 1) mma_commit(&bars->acc_full);
             }
-            if (bars->abort_flag != 0) {
+            __syncwarp();
+        }
+        if (__any_sync(0xffffffffu, bars->abort_flag != 0)) {
+            if (elect_one()) {
                 mma_commit(&bars->drain);
                 mbar_wait_drain(&bars->drain, 0);
             }
@@ -469,18 +477,19 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         }
         __syncwarp();
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);  // S^T = K Q^T, dP^T = V dO^T
-            constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);       // dV += P^T dO, dK += dS^T Q
-            const uint32_t dK = desc_lo_k_major(smem_u32(sK)), dV = desc_lo_k_major(smem_u32(sV));
-            auto issue_scores = [&](int it) -> bool {
-                const int st = it % C::kStages;
-                if (!mbar_wait(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 2)) return false;
-                tc_fence_after();
-                const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
-                const uint32_t dQ = desc_lo_k_major(aQ), dDO = desc_lo_k_major(aQ + C::kSubTileBytes);
-                const uint32_t tS = tmem_base + kColS + (it & 1) * kSubTile;
-                const uint32_t tP = tmem_base + kColP + (it & 1) * kSubTile;
+        // Warp-uniform loop, one elected lane issues (see the dQ kernel).
+        constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);  // S^T = K Q^T, dP^T = V dO^T
+        constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);       // dV += P^T dO, dK += dS^T Q
+        const uint32_t dK = desc_lo_k_major(smem_u32(sK)), dV = desc_lo_k_major(smem_u32(sV));
+        auto issue_scores = [&](int it) -> bool {
+            const int st = it % C::kStages;
+            if (!mbar_wait_uniform(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 2)) return false;
+            tc_fence_after();
+            const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
+            const uint32_t dQ = desc_lo_k_major(aQ), dDO = desc_lo_k_major(aQ + C::kSubTileBytes);
+            const uint32_t tS = tmem_base + kColS + (it & 1) * kSubTile;
+            const uint32_t tP = tmem_base + kColP + (it & 1) * kSubTile;
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk)
                     mma_ss(tS, dK + desc_step_k_major(kk, C::kBigBoxBytes), dQ + desc_step_k_major(kk, C::kSubBoxBytes),
@@ -490,20 +499,23 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                     mma_ss(tP, dV + desc_step_k_major(kk, C::kBigBoxBytes), dDO + desc_step_k_major(kk, C::kSubBoxBytes),
                            idesc_sc, kk > 0);
                 mma_commit(&bars->s_full[it & 1]);
-                return true;
-            };
-            bool ok = mbar_wait(&bars->res_full, 0, ctx, kWaitBwdDkDv + 3);
-            ok = ok && issue_scores(0);
-            for (int it = 0; ok && it < total_steps; ++it) {
-                if (it + 1 < total_steps && !issue_scores(it + 1)) break;
-                if (!mbar_wait(&bars->p_full[it & 1], (it >> 1) & 1, ctx, kWaitBwdDkDv + 4)) break;
-                tc_fence_after();
-                const int st = it % C::kStages;
-                const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
-                const uint32_t dQmn = desc_lo_mn_major(aQ, C::kSubBoxBytes);
-                const uint32_t dDOmn = desc_lo_mn_major(aQ + C::kSubTileBytes, C::kSubBoxBytes);
-                const uint32_t tPt = tmem_base + kColS + (it & 1) * kSubTile;   // bf16 P^T over the S^T buffer
-                const uint32_t tdSt = tmem_base + kColP + (it & 1) * kSubTile;  // bf16 dS^T over the dP^T buffer
+            }
+            __syncwarp();
+            return true;
+        };
+        bool ok = mbar_wait_uniform(&bars->res_full, 0, ctx, kWaitBwdDkDv + 3);
+        ok = ok && issue_scores(0);
+        for (int it = 0; ok && it < total_steps; ++it) {
+            if (it + 1 < total_steps && !issue_scores(it + 1)) break;
+            if (!mbar_wait_uniform(&bars->p_full[it & 1], (it >> 1) & 1, ctx, kWaitBwdDkDv + 4)) break;
+            tc_fence_after();
+            const int st = it % C::kStages;
+            const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
+            const uint32_t dQmn = desc_lo_mn_major(aQ, C::kSubBoxBytes);
+            const uint32_t dDOmn = desc_lo_mn_major(aQ + C::kSubTileBytes, C::kSubBoxBytes);
+            const uint32_t tPt = tmem_base + kColS + (it & 1) * kSubTile;   // bf16 P^T over the S^T buffer
+            const uint32_t tdSt = tmem_base + kColP + (it & 1) * kSubTile;  // bf16 dS^T over the dP^T buffer
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kSubTile / 16; ++kk)
                     mma_ts(tmem_base + kColDV, tPt + packed_operand_col(kk), dDOmn + kk * kDescStepMn, idesc_acc,
@@ -515,7 +527,10 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                 mma_commit(&bars->st_empty[st]);
                 if (it == total_steps - 1) mma_commit(&bars->acc_full);
             }
-            if (bars->abort_flag != 0) {
+            __syncwarp();
+        }
+        if (__any_sync(0xffffffffu, bars->abort_flag != 0)) {
+            if (elect_one()) {
                 mma_commit(&bars->drain);
                 mbar_wait_drain(&bars->drain, 0);
             }

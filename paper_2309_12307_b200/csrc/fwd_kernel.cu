@@ -153,22 +153,24 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
         __syncwarp();
     } else if (warp == 1) {
         // =========================== MMA issuer ==============================================
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);  // S = Q K^T   (both K-major)
-            constexpr uint32_t idesc_o = idesc_bf16(128, HD, 0, 1);   // O += P V    (V is MN-major)
-            const uint32_t tS = tmem_base + C::kColS;
-            const uint32_t tO = tmem_base + C::kColO;
-            const uint32_t dQ = desc_lo_k_major(smem_u32(sQ));
-            bool ok = mbar_wait(q_full, 0, ctx, kWaitFwd + 3);
-            for (int j = 0; ok && j < n_kv; ++j) {
-                const int st = j % C::kStages;
-                const uint32_t ph = (j / C::kStages) & 1;
-                const uint32_t dK = desc_lo_k_major(smem_u32(sK + st * C::kTileBytes));
-                const uint32_t dV = desc_lo_mn_major(smem_u32(sV + st * C::kTileBytes), C::kBoxBytes);
-                if (!mbar_wait(k_full + st, ph, ctx, kWaitFwd + 4)) break;
-                tc_fence_after();
-                // The previous P (aliased on S) was consumed by the previous P.V, which precedes
-                // this MMA in issue order; the softmax warps finished reading S before that.
+        // The whole warp walks the loop so that addresses and descriptors stay warp-uniform values;
+        // only the MMA and commit instructions themselves are issued by one elected lane.
+        constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);  // S = Q K^T   (both K-major)
+        constexpr uint32_t idesc_o = idesc_bf16(128, HD, 0, 1);   // O += P V    (V is MN-major)
+        const uint32_t tS = tmem_base + C::kColS;
+        const uint32_t tO = tmem_base + C::kColO;
+        const uint32_t dQ = desc_lo_k_major(smem_u32(sQ));
+        bool ok = mbar_wait_uniform(q_full, 0, ctx, kWaitFwd + 3);
+        for (int j = 0; ok && j < n_kv; ++j) {
+            const int st = j % C::kStages;
+            const uint32_t ph = (j / C::kStages) & 1;
+            const uint32_t dK = desc_lo_k_major(smem_u32(sK + st * C::kTileBytes));
+            const uint32_t dV = desc_lo_mn_major(smem_u32(sV + st * C::kTileBytes), C::kBoxBytes);
+            if (!mbar_wait_uniform(k_full + st, ph, ctx, kWaitFwd + 4)) break;
+            tc_fence_after();
+            // The previous P (aliased on S) was consumed by the previous P.V, which precedes
+            // this MMA in issue order; the softmax warps finished reading S before that.
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
                     constexpr uint32_t kBox = C::kBoxBytes;
@@ -176,9 +178,12 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
                 }
                 mma_commit(k_empty + st);
                 mma_commit(s_full);
-                if (!mbar_wait(p_full, j & 1, ctx, kWaitFwd + 5)) break;
-                if (!mbar_wait(v_full + st, ph, ctx, kWaitFwd + 6)) break;
-                tc_fence_after();
+            }
+            __syncwarp();
+            if (!mbar_wait_uniform(p_full, j & 1, ctx, kWaitFwd + 5)) break;
+            if (!mbar_wait_uniform(v_full + st, ph, ctx, kWaitFwd + 6)) break;
+            tc_fence_after();
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kTile / 16; ++kk) {
                     mma_ts(tO, tS + (kk >> 2) * 64 + (kk & 3) * 8, dV + kk * kDescStepMn, idesc_o, (j > 0) || (kk > 0));
@@ -186,8 +191,11 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
                 mma_commit(v_empty + st);
                 if (j == n_kv - 1) mma_commit(o_full);
             }
-            if (*abort_flag != 0) {
-                // MMAs already issued must finish before tensor memory is released
+            __syncwarp();
+        }
+        if (__any_sync(0xffffffffu, *abort_flag != 0)) {
+            // MMAs already issued must finish before tensor memory is released
+            if (elect_one()) {
                 mma_commit(drain);
                 mbar_wait_drain(drain, 0);
             }

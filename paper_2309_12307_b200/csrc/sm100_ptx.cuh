@@ -76,6 +76,24 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const 
     }
     return true;
 }
+// All 32 lanes wait; the outcome is made warp-uniform so the warp can keep executing warp-wide
+// instructions (or leave its loop) together.
+__device__ __forceinline__ bool mbar_wait_uniform(uint64_t* bar, uint32_t parity, const WaitCtx& ctx, int where) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, ctx, where) ? 1 : 0) != 0;
+}
+// One lane of a fully active warp (the same lane every time for a given warp).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "elect.sync _|p, 0xffffffff;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 // Teardown helper for an aborting CTA: wait (time-limited, ignoring the abort flag) for an
 // operation that is still in flight so that it cannot land after the CTA's resources are reused.
 __device__ __forceinline__ void mbar_wait_drain(uint64_t* bar, uint32_t parity) {

@@ -14,11 +14,12 @@
 // The roll of the shifted heads and the group boundaries are folded into TMA coordinates exactly
 // as in the forward kernel; all results are stored at original token rows.
 //
-// Both tensor-core kernels share one software pipeline (320 threads, one CTA per SM): warp 0
-// loads with TMA, warp 1 issues tcgen05 MMAs, warps 2-9 do the elementwise work with one
-// tensor-memory lane and half of the columns per thread.  The two score products of step n+1 are issued before the
-// gradient products of step n, into the other half of a double buffer, so the elementwise work
-// of step n overlaps tensor-core work.
+// Both tensor-core kernels share one software pipeline (384 threads, one CTA per SM): warp 0
+// loads with TMA; warp 1 issues the score MMAs and warp 2 the gradient MMAs (a single issuing
+// warp spends so long on its own barrier waits that the tensor pipe runs dry in between; with two,
+// one can issue while the other waits); warps 4-11 do the elementwise work with one tensor-memory
+// lane and half of the columns per thread.  Score buffers are double-buffered, so the score
+// products of step n+1 run while the elementwise warps work on step n.
 #include "s2a_params.h"
 #include "sm100_ptx.cuh"
 
@@ -73,7 +74,7 @@ __global__ void __launch_bounds__(256) s2a_bwd_preprocess_kernel(const PreParams
 // ------------------------------------------------------------------------------------------------
 template <int HD>
 struct BwdCfg {
-    static constexpr int kThreads = 320;  // TMA warp, MMA warp, 8 elementwise warps
+    static constexpr int kThreads = 384;  // TMA warp, two MMA warps, one spare, 8 elementwise warps
     static constexpr int kBoxes = HD / 64;
     static constexpr int kBigBoxBytes = kTile * 128;            // 128-row box
     static constexpr int kSubBoxBytes = kSubTile * 128;         // 64-row box
@@ -128,9 +129,11 @@ template <int kStages>
 struct BwdBars {
     uint64_t res_full;            // resident operands landed
     uint64_t acc_full;            // all gradient MMAs done
-    uint64_t drain;               // abort path only
+    uint64_t drain;               // abort path only (gradient MMA warp)
+    uint64_t drain2;              // abort path only (score MMA warp)
     uint64_t s_full[2];           // score products of a step are in tensor memory
     uint64_t p_full[2];           // bf16 P / dS of a step are in tensor memory
+    uint64_t buf_free[2];         // gradient MMAs that read a score buffer's bf16 operands are done
     uint64_t st_full[kStages];    // streamed operands of a stage landed
     uint64_t st_empty[kStages];   // MMAs reading a stage are done
     uint32_t tmem_slot;
@@ -178,9 +181,11 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         mbar_init(&bars->res_full, 1);
         mbar_init(&bars->acc_full, 1);
         mbar_init(&bars->drain, 1);
+        mbar_init(&bars->drain2, 1);
         for (int x = 0; x < 2; ++x) {
             mbar_init(&bars->s_full[x], 1);
             mbar_init(&bars->p_full[x], 256);
+            mbar_init(&bars->buf_free[x], 1);
         }
         for (int st = 0; st < C::kStages; ++st) {
             mbar_init(&bars->st_full[st], 1);
@@ -193,7 +198,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         tma_prefetch_desc(&p.tm_k);
         tma_prefetch_desc(&p.tm_v);
     }
-    if (warp == 1) {
+    if (warp == 3) {
         tmem_alloc(&bars->tmem_slot, C::kTmemCols);
         tmem_relinquish();
     }
@@ -233,15 +238,17 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         }
         __syncwarp();
     } else if (warp == 1) {
-        // The whole warp walks the loop so that addresses and descriptors stay warp-uniform values;
-        // only the MMA and commit instructions themselves are issued by one elected lane.
-        constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);  // S = Q K^T, dP = dO V^T
-        constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);       // dQ += dS K   (K is MN-major)
+        // ---- score MMAs: S = Q K^T and dP = dO V^T of step n into buffer n & 1.  The whole warp
+        // walks the loop so that addresses and descriptors stay warp-uniform values; only the MMA
+        // and commit instructions themselves are issued by one elected lane.
+        constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);
         const uint32_t dQ = desc_lo_k_major(smem_u32(sQ)), dDO = desc_lo_k_major(smem_u32(sDO));
-        // score products of step n into buffer n & 1
-        auto issue_scores = [&](int n) -> bool {
+        bool ok = mbar_wait_uniform(&bars->res_full, 0, ctx, kWaitBwdDq + 3);
+        for (int n = 0; ok && n < n_steps; ++n) {
             const int st = n % C::kStages;
-            if (!mbar_wait_uniform(&bars->st_full[st], (n / C::kStages) & 1, ctx, kWaitBwdDq + 2)) return false;
+            if (!mbar_wait_uniform(&bars->st_full[st], (n / C::kStages) & 1, ctx, kWaitBwdDq + 2)) break;
+            // buffer n & 1 still holds the bf16 dS of step n - 2 until that step's dQ MMAs are done
+            if (n >= 2 && !mbar_wait_uniform(&bars->buf_free[n & 1], ((n - 2) >> 1) & 1, ctx, kWaitBwdDq + 7)) break;
             tc_fence_after();
             const uint32_t aK = smem_u32(sStage + st * C::kStageBytes);
             const uint32_t dK = desc_lo_k_major(aK), dV = desc_lo_k_major(aK + C::kSubTileBytes);
@@ -259,15 +266,21 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
                 mma_commit(&bars->s_full[n & 1]);
             }
             __syncwarp();
-            return true;
-        };
-        bool ok = mbar_wait_uniform(&bars->res_full, 0, ctx, kWaitBwdDq + 3);
-        ok = ok && issue_scores(0);
-        for (int n = 0; ok && n < n_steps; ++n) {
-            if (n + 1 < n_steps && !issue_scores(n + 1)) break;
+        }
+        if (__any_sync(0xffffffffu, bars->abort_flag != 0)) {
+            if (elect_one()) {
+                mma_commit(&bars->drain2);
+                mbar_wait_drain(&bars->drain2, 0);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 2) {
+        // ---- gradient MMAs: dQ += dS K of step n (K is MN-major in the tile that served Q K^T)
+        constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);
+        for (int n = 0; n < n_steps; ++n) {
+            const int st = n % C::kStages;
             if (!mbar_wait_uniform(&bars->p_full[n & 1], (n >> 1) & 1, ctx, kWaitBwdDq + 4)) break;
             tc_fence_after();
-            const int st = n % C::kStages;
             const uint32_t dKmn = desc_lo_mn_major(smem_u32(sStage + st * C::kStageBytes), C::kSubBoxBytes);
             const uint32_t tdS = tmem_base + kColS + (n & 1) * kSubTile;  // bf16 dS over the S buffer
             if (elect_one()) {
@@ -276,20 +289,24 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
                     mma_ts(tmem_base + kColAcc, tdS + packed_operand_col(kk), dKmn + kk * kDescStepMn, idesc_acc,
                            (n > 0) || (kk > 0));
                 mma_commit(&bars->st_empty[st]);
+                mma_commit(&bars->buf_free[n & 1]);
                 if (n == n_steps - 1) mma_commit(&bars->acc_full);
             }
             __syncwarp();
         }
         if (__any_sync(0xffffffffu, bars->abort_flag != 0)) {
+            // MMAs already issued (by either MMA warp) must finish before tensor memory is released
             if (elect_one()) {
                 mma_commit(&bars->drain);
                 mbar_wait_drain(&bars->drain, 0);
             }
         }
         __syncwarp();
+    } else if (warp == 3) {
+        // spare warp: owns the tensor-memory allocation only
     } else {
         const int quad = warp & 3;
-        const int half = (warp - 2) >> 2;
+        const int half = (warp - 4) >> 2;
         const int row = quad * 32 + lane;
         const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
         const size_t stat_idx = (static_cast<size_t>(b) * geo.H + h) * geo.N + tq0 + row;
@@ -306,9 +323,10 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
             tmem_ld_32x32(tS, sr);
             tmem_ld_32x32(tP, pr);
             tmem_wait_ld();
-            float ds[32];
+            uint32_t pk[16];
             if (n >= 2 * i) {
                 // diagonal sub-tiles: key x is visible to query row r iff 64 n + x <= 128 i + r
+                float ds[32];
                 const int lim = i * kTile + row - n * kSubTile - half * 32;  // visible iff e <= lim
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
@@ -316,15 +334,22 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
                     if (e > lim) pe = 0.f;
                     ds[e] = pe * (__uint_as_float(pr[e]) - Drow);
                 }
+                pack32(ds, pk);
             } else {
+                // two columns per instruction for the multiply-adds
+                const uint64_t c2x2 = f2_pack(c2, c2), nlx2 = f2_pack(neg_lse2, neg_lse2), Dx2 = f2_pack(Drow, Drow);
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, neg_lse2));
-                    ds[e] = pe * (__uint_as_float(pr[e]) - Drow);
+                for (int e = 0; e < 16; ++e) {
+                    const uint64_t x = f2_fma(f2_pack(__uint_as_float(sr[2 * e]), __uint_as_float(sr[2 * e + 1])), c2x2, nlx2);
+                    float x0, x1;
+                    f2_unpack(x, x0, x1);
+                    const uint64_t pe = f2_pack(fast_exp2(x0), fast_exp2(x1));
+                    const uint64_t t = f2_sub(f2_pack(__uint_as_float(pr[2 * e]), __uint_as_float(pr[2 * e + 1])), Dx2);
+                    float d0, d1;
+                    f2_unpack(f2_mul(pe, t), d0, d1);
+                    pk[e] = pack_bf16(d0, d1);
                 }
             }
-            uint32_t pk[16];
-            pack32(ds, pk);
             tmem_st_32x16(tS, pk);
             tmem_wait_st();
             tc_fence_before();
@@ -339,7 +364,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == 3) {
         tc_fence_after();
         tmem_dealloc(tmem_base, C::kTmemCols);
     }
@@ -414,9 +439,11 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         mbar_init(&bars->res_full, 1);
         mbar_init(&bars->acc_full, 1);
         mbar_init(&bars->drain, 1);
+        mbar_init(&bars->drain2, 1);
         for (int x = 0; x < 2; ++x) {
             mbar_init(&bars->s_full[x], 1);
             mbar_init(&bars->p_full[x], 256);
+            mbar_init(&bars->buf_free[x], 1);
         }
         for (int st = 0; st < C::kStages; ++st) {
             mbar_init(&bars->st_full[st], 1);
@@ -429,7 +456,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         tma_prefetch_desc(&p.tm_k);
         tma_prefetch_desc(&p.tm_v);
     }
-    if (warp == 1) {
+    if (warp == 3) {
         tmem_alloc(&bars->tmem_slot, C::kTmemCols);
         tmem_relinquish();
     }
@@ -477,13 +504,15 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         }
         __syncwarp();
     } else if (warp == 1) {
-        // Warp-uniform loop, one elected lane issues (see the dQ kernel).
-        constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);  // S^T = K Q^T, dP^T = V dO^T
-        constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);       // dV += P^T dO, dK += dS^T Q
+        // ---- score MMAs: S^T = K Q^T and dP^T = V dO^T of step `it` into buffer it & 1
+        // (warp-uniform loop, one elected lane issues; see the dQ kernel)
+        constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);
         const uint32_t dK = desc_lo_k_major(smem_u32(sK)), dV = desc_lo_k_major(smem_u32(sV));
-        auto issue_scores = [&](int it) -> bool {
+        bool ok = mbar_wait_uniform(&bars->res_full, 0, ctx, kWaitBwdDkDv + 3);
+        for (int it = 0; ok && it < total_steps; ++it) {
             const int st = it % C::kStages;
-            if (!mbar_wait_uniform(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 2)) return false;
+            if (!mbar_wait_uniform(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 2)) break;
+            if (it >= 2 && !mbar_wait_uniform(&bars->buf_free[it & 1], ((it - 2) >> 1) & 1, ctx, kWaitBwdDkDv + 8)) break;
             tc_fence_after();
             const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
             const uint32_t dQ = desc_lo_k_major(aQ), dDO = desc_lo_k_major(aQ + C::kSubTileBytes);
@@ -501,15 +530,21 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                 mma_commit(&bars->s_full[it & 1]);
             }
             __syncwarp();
-            return true;
-        };
-        bool ok = mbar_wait_uniform(&bars->res_full, 0, ctx, kWaitBwdDkDv + 3);
-        ok = ok && issue_scores(0);
-        for (int it = 0; ok && it < total_steps; ++it) {
-            if (it + 1 < total_steps && !issue_scores(it + 1)) break;
+        }
+        if (__any_sync(0xffffffffu, bars->abort_flag != 0)) {
+            if (elect_one()) {
+                mma_commit(&bars->drain2);
+                mbar_wait_drain(&bars->drain2, 0);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 2) {
+        // ---- gradient MMAs: dV += P^T dO and dK += dS^T Q of step `it`
+        constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);
+        for (int it = 0; it < total_steps; ++it) {
+            const int st = it % C::kStages;
             if (!mbar_wait_uniform(&bars->p_full[it & 1], (it >> 1) & 1, ctx, kWaitBwdDkDv + 4)) break;
             tc_fence_after();
-            const int st = it % C::kStages;
             const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
             const uint32_t dQmn = desc_lo_mn_major(aQ, C::kSubBoxBytes);
             const uint32_t dDOmn = desc_lo_mn_major(aQ + C::kSubTileBytes, C::kSubBoxBytes);
@@ -525,6 +560,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                     mma_ts(tmem_base + kColDK, tdSt + packed_operand_col(kk), dQmn + kk * kDescStepMn, idesc_acc,
                            (it > 0) || (kk > 0));
                 mma_commit(&bars->st_empty[st]);
+                mma_commit(&bars->buf_free[it & 1]);
                 if (it == total_steps - 1) mma_commit(&bars->acc_full);
             }
             __syncwarp();
@@ -536,9 +572,11 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
             }
         }
         __syncwarp();
+    } else if (warp == 3) {
+        // spare warp: owns the tensor-memory allocation only
     } else {
         const int quad = warp & 3;
-        const int half = (warp - 2) >> 2;
+        const int half = (warp - 4) >> 2;
         const int row = quad * 32 + lane;  // key row of the tile owned by this thread
         const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
         const float c2 = p.scale_log2;
@@ -560,30 +598,56 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                 tmem_ld_32x32(tS, sr);
                 tmem_ld_32x32(tP, pr);
                 tmem_wait_ld();
-                float pt[32], ds[32];
+                uint32_t pkP[16], pkS[16];
                 // query x of this sub-tile sees key row r iff 128 j + r <= 64 n + x
-                const bool diagonal = n < w.n_begin + 2;
-                const int lim = diagonal ? w.j * kTile + row - n * kSubTile - half * 32 : -1;  // visible iff e >= lim
+                if (n < w.n_begin + 2) {
+                    // diagonal sub-tiles: scalar path with the mask
+                    const int lim = w.j * kTile + row - n * kSubTile - half * 32;  // visible iff e >= lim
+                    float pt[32], ds[32];
 #pragma unroll
-                for (int e4 = 0; e4 < 8; ++e4) {
-                    const float4 l = lse4[e4];
-                    const float4 dd = d4[e4];
-                    const float lv[4] = {l.x, l.y, l.z, l.w};
-                    const float dv[4] = {dd.x, dd.y, dd.z, dd.w};
+                    for (int e4 = 0; e4 < 8; ++e4) {
+                        const float4 l = lse4[e4];
+                        const float4 dd = d4[e4];
+                        const float lv[4] = {l.x, l.y, l.z, l.w};
+                        const float dv[4] = {dd.x, dd.y, dd.z, dd.w};
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int e = e4 * 4 + u;
-                        float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, -lv[u] * kLog2e));
-                        if (diagonal && e < lim) pe = 0.f;
-                        pt[e] = pe;
-                        ds[e] = pe * (__uint_as_float(pr[e]) - dv[u]);
+                        for (int u = 0; u < 4; ++u) {
+                            const int e = e4 * 4 + u;
+                            float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, -lv[u] * kLog2e));
+                            if (e < lim) pe = 0.f;
+                            pt[e] = pe;
+                            ds[e] = pe * (__uint_as_float(pr[e]) - dv[u]);
+                        }
+                    }
+                    pack32(pt, pkP);
+                    pack32(ds, pkS);
+                } else {
+                    // two columns per instruction for the multiply-adds
+                    const uint64_t c2x2 = f2_pack(c2, c2), nl2e = f2_pack(-kLog2e, -kLog2e);
+#pragma unroll
+                    for (int e4 = 0; e4 < 8; ++e4) {
+                        const float4 l = lse4[e4];
+                        const float4 dd = d4[e4];
+                        const uint64_t lp[2] = {f2_pack(l.x, l.y), f2_pack(l.z, l.w)};
+                        const uint64_t dp[2] = {f2_pack(dd.x, dd.y), f2_pack(dd.z, dd.w)};
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const int e = e4 * 4 + 2 * u;
+                            const uint64_t x = f2_fma(f2_pack(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), c2x2,
+                                                      f2_mul(lp[u], nl2e));
+                            float x0, x1;
+                            f2_unpack(x, x0, x1);
+                            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                            pkP[e >> 1] = pack_bf16(p0, p1);
+                            const uint64_t t = f2_sub(f2_pack(__uint_as_float(pr[e]), __uint_as_float(pr[e + 1])), dp[u]);
+                            float d0, d1;
+                            f2_unpack(f2_mul(f2_pack(p0, p1), t), d0, d1);
+                            pkS[e >> 1] = pack_bf16(d0, d1);
+                        }
                     }
                 }
-                uint32_t pk[16];
-                pack32(pt, pk);
-                tmem_st_32x16(tS, pk);
-                pack32(ds, pk);
-                tmem_st_32x16(tP, pk);
+                tmem_st_32x16(tS, pkP);
+                tmem_st_32x16(tP, pkS);
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(&bars->p_full[it & 1]);
@@ -599,7 +663,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == 3) {
         tc_fence_after();
         tmem_dealloc(tmem_base, C::kTmemCols);
     }

@@ -590,8 +590,14 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                 if (!mbar_wait(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 5)) { ok = false; break; }
                 if (!mbar_wait(&bars->s_full[it & 1], (it >> 1) & 1, ctx, kWaitBwdDkDv + 6)) { ok = false; break; }
                 tc_fence_after();
-                const float4* lse4 = reinterpret_cast<const float4*>(sStat + st * 2 * kSubTile) + half * 8;
-                const float4* d4 = lse4 + kSubTile / 4;
+                // lse[64] then D[64] of this stage; this thread's 32 columns start at float 32 * half.
+                // (explicit shared-memory loads: through a generic pointer they cost far more latency)
+                const uint32_t stat_sa = smem_u32(sStat + st * 2 * kSubTile) + half * 128;
+                auto lds4 = [](uint32_t a) {
+                    float4 r;
+                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(a));
+                    return r;
+                };
                 const uint32_t tS = t_row + kColS + (it & 1) * kSubTile + half * 32;
                 const uint32_t tP = t_row + kColP + (it & 1) * kSubTile + half * 32;
                 uint32_t sr[32], pr[32];
@@ -606,8 +612,8 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                     float pt[32], ds[32];
 #pragma unroll
                     for (int e4 = 0; e4 < 8; ++e4) {
-                        const float4 l = lse4[e4];
-                        const float4 dd = d4[e4];
+                        const float4 l = lds4(stat_sa + e4 * 16);
+                        const float4 dd = lds4(stat_sa + kSubTile * 4 + e4 * 16);
                         const float lv[4] = {l.x, l.y, l.z, l.w};
                         const float dv[4] = {dd.x, dd.y, dd.z, dd.w};
 #pragma unroll
@@ -626,8 +632,8 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                     const uint64_t c2x2 = f2_pack(c2, c2), nl2e = f2_pack(-kLog2e, -kLog2e);
 #pragma unroll
                     for (int e4 = 0; e4 < 8; ++e4) {
-                        const float4 l = lse4[e4];
-                        const float4 dd = d4[e4];
+                        const float4 l = lds4(stat_sa + e4 * 16);
+                        const float4 dd = lds4(stat_sa + kSubTile * 4 + e4 * 16);
                         const uint64_t lp[2] = {f2_pack(l.x, l.y), f2_pack(l.z, l.w)};
                         const uint64_t dp[2] = {f2_pack(dd.x, dd.y), f2_pack(dd.z, dd.w)};
 #pragma unroll

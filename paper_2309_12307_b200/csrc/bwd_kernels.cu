@@ -131,9 +131,9 @@ struct BwdBars {
     uint64_t acc_full;            // all gradient MMAs done
     uint64_t drain;               // abort path only (gradient MMA warp)
     uint64_t drain2;              // abort path only (score MMA warp)
-    uint64_t s_full[2];           // score products of a step are in tensor memory
-    uint64_t p_full[2];           // bf16 P / dS of a step are in tensor memory
-    uint64_t buf_free[2];         // gradient MMAs that read a score buffer's bf16 operands are done
+    uint64_t s_full[3];           // score products of a step are in tensor memory
+    uint64_t p_full[3];           // bf16 P / dS of a step are in tensor memory
+    uint64_t buf_free[3];         // gradient MMAs that read a score buffer's bf16 operands are done
     uint64_t st_full[kStages];    // streamed operands of a stage landed
     uint64_t st_empty[kStages];   // MMAs reading a stage are done
     uint32_t tmem_slot;
@@ -143,11 +143,14 @@ struct BwdBars {
 // ------------------------------------------------------------------------------------------------
 // 2. dQ
 // ------------------------------------------------------------------------------------------------
-// Tensor memory columns: dQ [0,HD)   S buffers [128,192) [192,256)   dP buffers [256,320) [320,384)
+// Tensor memory columns: dQ [0,HD)   three S buffers [128,320)   three dP buffers [320,512)
+// (three score buffers in flight: the chain scores -> elementwise -> dQ MMA of one buffer is about
+// twice as long as the tensor-pipe work of a step, so two buffers leave the pipe idle)
 template <int HD>
 __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(const __grid_constant__ BwdDqParams p) {
     using C = BwdCfg<HD>;
     using Bars = BwdBars<C::kStages>;
+    constexpr int kBufs = 3;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem;                                // resident: Q_i
@@ -182,7 +185,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         mbar_init(&bars->acc_full, 1);
         mbar_init(&bars->drain, 1);
         mbar_init(&bars->drain2, 1);
-        for (int x = 0; x < 2; ++x) {
+        for (int x = 0; x < kBufs; ++x) {
             mbar_init(&bars->s_full[x], 1);
             mbar_init(&bars->p_full[x], 256);
             mbar_init(&bars->buf_free[x], 1);
@@ -207,7 +210,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_slot;
     const WaitCtx ctx{&bars->abort_flag, p.status};
-    constexpr uint32_t kColAcc = 0, kColS = 128, kColP = 256;
+    constexpr uint32_t kColAcc = 0, kColS = 128, kColP = 128 + kBufs * kSubTile;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -238,7 +241,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ---- score MMAs: S = Q K^T and dP = dO V^T of step n into buffer n & 1.  The whole warp
+        // ---- score MMAs: S = Q K^T and dP = dO V^T of step n into buffer n % 3.  The whole warp
         // walks the loop so that addresses and descriptors stay warp-uniform values; only the MMA
         // and commit instructions themselves are issued by one elected lane.
         constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);
@@ -247,13 +250,15 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         for (int n = 0; ok && n < n_steps; ++n) {
             const int st = n % C::kStages;
             if (!mbar_wait_uniform(&bars->st_full[st], (n / C::kStages) & 1, ctx, kWaitBwdDq + 2)) break;
-            // buffer n & 1 still holds the bf16 dS of step n - 2 until that step's dQ MMAs are done
-            if (n >= 2 && !mbar_wait_uniform(&bars->buf_free[n & 1], ((n - 2) >> 1) & 1, ctx, kWaitBwdDq + 7)) break;
+            const int bf = n % kBufs;
+            const uint32_t use = (n / kBufs) & 1;  // parity of this buffer's use count
+            // the buffer still holds the bf16 dS of step n - 3 until that step's dQ MMAs are done
+            if (n >= kBufs && !mbar_wait_uniform(&bars->buf_free[bf], use ^ 1, ctx, kWaitBwdDq + 7)) break;
             tc_fence_after();
             const uint32_t aK = smem_u32(sStage + st * C::kStageBytes);
             const uint32_t dK = desc_lo_k_major(aK), dV = desc_lo_k_major(aK + C::kSubTileBytes);
-            const uint32_t tS = tmem_base + kColS + (n & 1) * kSubTile;
-            const uint32_t tP = tmem_base + kColP + (n & 1) * kSubTile;
+            const uint32_t tS = tmem_base + kColS + bf * kSubTile;
+            const uint32_t tP = tmem_base + kColP + bf * kSubTile;
             if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk)
@@ -263,7 +268,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
                 for (int kk = 0; kk < HD / 16; ++kk)
                     mma_ss(tP, dDO + desc_step_k_major(kk, C::kBigBoxBytes), dV + desc_step_k_major(kk, C::kSubBoxBytes),
                            idesc_sc, kk > 0);
-                mma_commit(&bars->s_full[n & 1]);
+                mma_commit(&bars->s_full[bf]);
             }
             __syncwarp();
         }
@@ -279,17 +284,18 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);
         for (int n = 0; n < n_steps; ++n) {
             const int st = n % C::kStages;
-            if (!mbar_wait_uniform(&bars->p_full[n & 1], (n >> 1) & 1, ctx, kWaitBwdDq + 4)) break;
+            const int bf = n % kBufs;
+            if (!mbar_wait_uniform(&bars->p_full[bf], (n / kBufs) & 1, ctx, kWaitBwdDq + 4)) break;
             tc_fence_after();
             const uint32_t dKmn = desc_lo_mn_major(smem_u32(sStage + st * C::kStageBytes), C::kSubBoxBytes);
-            const uint32_t tdS = tmem_base + kColS + (n & 1) * kSubTile;  // bf16 dS over the S buffer
+            const uint32_t tdS = tmem_base + kColS + bf * kSubTile;  // bf16 dS over the S buffer
             if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kSubTile / 16; ++kk)
                     mma_ts(tmem_base + kColAcc, tdS + packed_operand_col(kk), dKmn + kk * kDescStepMn, idesc_acc,
                            (n > 0) || (kk > 0));
                 mma_commit(&bars->st_empty[st]);
-                mma_commit(&bars->buf_free[n & 1]);
+                mma_commit(&bars->buf_free[bf]);
                 if (n == n_steps - 1) mma_commit(&bars->acc_full);
             }
             __syncwarp();
@@ -315,10 +321,11 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         const float c2 = p.scale_log2;
         bool ok = true;
         for (int n = 0; n < n_steps; ++n) {
-            if (!mbar_wait(&bars->s_full[n & 1], (n >> 1) & 1, ctx, kWaitBwdDq + 5)) { ok = false; break; }
+            const int bf = n % kBufs;
+            if (!mbar_wait(&bars->s_full[bf], (n / kBufs) & 1, ctx, kWaitBwdDq + 5)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t tS = t_row + kColS + (n & 1) * kSubTile + half * 32;
-            const uint32_t tP = t_row + kColP + (n & 1) * kSubTile + half * 32;
+            const uint32_t tS = t_row + kColS + bf * kSubTile + half * 32;
+            const uint32_t tP = t_row + kColP + bf * kSubTile + half * 32;
             uint32_t sr[32], pr[32];
             tmem_ld_32x32(tS, sr);
             tmem_ld_32x32(tP, pr);
@@ -353,7 +360,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
             tmem_st_32x16(tS, pk);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(&bars->p_full[n & 1]);
+            mbar_arrive(&bars->p_full[bf]);
         }
         if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDq + 6)) {
             tc_fence_after();

@@ -204,6 +204,7 @@ def run_ours(args):
 
     from paper_2309_12307_b200 import binding as s2a
     from paper_2309_12307_b200.inputs import WORKLOADS, make_workload_inputs
+    from paper_2309_12307_b200.replicas import slowest_rank_ms, whole_job_rate
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -274,10 +275,7 @@ def run_ours(args):
     if rc != 0:
         raise RuntimeError(f"device status {rc} (wait code {where}) in the timed region")
 
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms_max = float(t.item())
+    total_ms_max = slowest_rank_ms(total_ms, dev)
     flops_step = w.flops_fwd_bwd
     value = world * flops_step * K / (total_ms_max * 1e-3) / 1e12
 
@@ -302,10 +300,7 @@ def run_ours(args):
         s2a.s2a_fwd_bwd_host(pin, host_out, dev_bufs, G, ws, stream=stream)
     e1.record(stream)
     barrier()
-    te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_value = world * flops_step * Ke / (float(te.item()) * 1e-3) / 1e12
+    e2e_value = whole_job_rate(flops_step * Ke, e0.elapsed_time(e1), dev) / 1e12
 
     if rank != 0:
         if world > 1:

@@ -30,6 +30,11 @@ METRIC = "S2-Attn fwd+bwd TFLOP/s (causal in-group FLOPs)"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "llama2_7b_32k"
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
+# DRAM bytes (read + write) per launch from the ncu capture summarised in
+# profiles/dram_traffic_llama2_7b_8k.md, taken on llama2_7b_8k; every tensor is touched once, so
+# traffic scales with B*N*(H+Hkv)*d.  Set an entry to None when its kernel changes after the capture.
+NCU_TRAFFIC_8K = {"fwd": 249.4e6, "bwd_preprocess": 135.2e6, "bwd_dkdv": 373.5e6, "bwd_dq": 320.8e6}
+NCU_TRAFFIC_8K_SIZE = 1 * 8192 * (32 + 32) * 128
 
 
 def load_peaks():
@@ -323,8 +328,11 @@ def run_ours(args):
     dom = max(names, key=lambda n: kernel_ms[n])
     peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
     achieved = kernels[dom]["algorithmic_tflops"]
+    traffic = NCU_TRAFFIC_8K.get(dom)
+    if traffic is not None:
+        traffic = traffic * (B * N * (H + Hkv) * d) / NCU_TRAFFIC_8K_SIZE
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": None,
+                "frac": achieved / peak, "traffic": traffic, "traffic_unit": "bytes per launch (ncu on 8k, scaled)",
                 "peak_source": f"{peak_src} bf16 sustained (burst {peaks.get('bf16_tflops')})",
                 "whole_step_frac": value / world / peak}
 

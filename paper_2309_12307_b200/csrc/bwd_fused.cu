@@ -26,7 +26,7 @@ namespace {
 
 constexpr float kLog2eF = 1.4426950408889634f;
 constexpr int kHD = 128;
-constexpr int kFThreads = 384;                 // TMA warp, MMA warp, two spare warps, 8 elementwise warps
+constexpr int kFThreads = 640;                 // TMA warp, MMA warp, two spare warps, 2 x 8 elementwise warps
 constexpr int kFBox = kTile * 128;             // one 64-column TMA box of 128 rows
 constexpr int kFTile = 2 * kFBox;              // a 128 x 128 bf16 tile
 constexpr int kFStages = 2;
@@ -43,7 +43,7 @@ static_assert(kFPayload <= kFSmemBytes, "shared memory layout too large");
 
 struct FusedBars {
     uint64_t res_full, acc_full, drain;
-    uint64_t s_full, dp_full, p_ready, ds_ready, dq_full, dq_drained;
+    uint64_t s_full, dp_full, p_ready, p_taken, ds_ready, ds_free, dq_full, dq_drained;
     uint64_t st_full[kFStages], st_empty[kFStages];
     uint32_t tmem_slot;
     int abort_flag;
@@ -53,6 +53,12 @@ struct FusedBars {
 __device__ __forceinline__ int mod_pos_f(int x, int n) {
     int r = x % n;
     return r < 0 ? r + n : r;
+}
+
+__device__ __forceinline__ float4 lds_f4(uint32_t saddr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(saddr));
+    return v;
 }
 
 // query tiles that attend key tile tk0 in head hq: tiles j .. Tg-1 of group g (rolled order)
@@ -121,6 +127,8 @@ __global__ void __launch_bounds__(kFThreads, 1) s2a_bwd_fused_kernel(const __gri
         mbar_init(&bars->s_full, 1);
         mbar_init(&bars->dp_full, 1);
         mbar_init(&bars->p_ready, 256);
+        mbar_init(&bars->p_taken, 256);
+        mbar_init(&bars->ds_free, 1);
         mbar_init(&bars->ds_ready, 256);
         mbar_init(&bars->dq_full, 1);
         mbar_init(&bars->dq_drained, 256);
@@ -186,8 +194,8 @@ __global__ void __launch_bounds__(kFThreads, 1) s2a_bwd_fused_kernel(const __gri
         // =========================== MMA issuer ==============================================
         // The whole warp walks the loop (warp-uniform addresses); one elected lane issues.  All five
         // products of a step come from this one warp, in an order that keeps tensor-memory reuse safe:
-        // S^T(n) follows dV(n-1) (which read P^T from the same columns), dP^T(n) follows the
-        // draining of dQ^T(n-1) (same columns).
+        //   S^T(n+1) after dV(n) (same columns hold P^T(n)) and after group B has copied P^T(n) out,
+        //   dP^T(n)  after the draining of dQ^T(n-1) (same columns).
         constexpr uint32_t idesc_kk = idesc_bf16(128, 128, 0, 0);   // both operands K-major
         constexpr uint32_t idesc_kn = idesc_bf16(128, 128, 0, 1);   // B MN-major
         constexpr uint32_t idesc_nn = idesc_bf16(128, 128, 1, 1);   // A and B MN-major
@@ -196,15 +204,11 @@ __global__ void __launch_bounds__(kFThreads, 1) s2a_bwd_fused_kernel(const __gri
         const uint32_t dK_mn = desc_lo_mn_major(aK, kFBox);
         const uint32_t dDS_k = desc_lo_k_major(aDS), dDS_mn = desc_lo_mn_major(aDS, kFBox);
         const uint32_t tS = tmem_base + kColS, tP2 = tmem_base + kColP2;
-        bool ok = mbar_wait_uniform(&bars->res_full, 0, ctx, kWaitBwdFused + 2);
-        for (int n = 0; ok && n < total_steps; ++n) {
+        auto issue_scores = [&](int n) -> bool {   // S^T(n) = K Q(n)^T
             const int st = n % kFStages;
-            const uint32_t par = n & 1;
-            const uint32_t aQ = smem_u32(sStage + st * 2 * kFTile), aDO = aQ + kFTile;
-            const uint32_t dQ_k = desc_lo_k_major(aQ), dDO_k = desc_lo_k_major(aDO);
-            const uint32_t dQ_mn = desc_lo_mn_major(aQ, kFBox), dDO_mn = desc_lo_mn_major(aDO, kFBox);
-            if (!mbar_wait_uniform(&bars->st_full[st], (n / kFStages) & 1, ctx, kWaitBwdFused + 3)) break;
+            if (!mbar_wait_uniform(&bars->st_full[st], (n / kFStages) & 1, ctx, kWaitBwdFused + 3)) return false;
             tc_fence_after();
+            const uint32_t dQ_k = desc_lo_k_major(smem_u32(sStage + st * 2 * kFTile));
             if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
@@ -212,6 +216,16 @@ __global__ void __launch_bounds__(kFThreads, 1) s2a_bwd_fused_kernel(const __gri
                 mma_commit(&bars->s_full);
             }
             __syncwarp();
+            return true;
+        };
+        bool ok = mbar_wait_uniform(&bars->res_full, 0, ctx, kWaitBwdFused + 2);
+        ok = ok && issue_scores(0);
+        for (int n = 0; ok && n < total_steps; ++n) {
+            const int st = n % kFStages;
+            const uint32_t par = n & 1;
+            const uint32_t aQ = smem_u32(sStage + st * 2 * kFTile), aDO = aQ + kFTile;
+            const uint32_t dDO_k = desc_lo_k_major(aDO);
+            const uint32_t dQ_mn = desc_lo_mn_major(aQ, kFBox), dDO_mn = desc_lo_mn_major(aDO, kFBox);
             if (n > 0 && !mbar_wait_uniform(&bars->dq_drained, par ^ 1, ctx, kWaitBwdFused + 4)) break;
             tc_fence_after();
             if (elect_one()) {
@@ -230,17 +244,24 @@ __global__ void __launch_bounds__(kFThreads, 1) s2a_bwd_fused_kernel(const __gri
                            (n > 0) || (kk > 0));
             }
             __syncwarp();
+            if (n + 1 < total_steps) {
+                // the next scores overwrite P^T(n): dV(n) precedes them in issue order, and group B must have
+                // taken its copy of P^T(n)
+                if (!mbar_wait_uniform(&bars->p_taken, par, ctx, kWaitBwdFused + 12)) break;
+                if (!issue_scores(n + 1)) break;
+            }
             if (!mbar_wait_uniform(&bars->ds_ready, par, ctx, kWaitBwdFused + 6)) break;
             tc_fence_after();
             if (elect_one()) {
 #pragma unroll
+                for (int kk = 0; kk < 8; ++kk)   // dQ^T = K^T dS^T first: its columns have to be drained before the next dP^T
+                    mma_ss(tP2, dK_mn + kk * kDescStepMn, dDS_mn + kk * kDescStepMn, idesc_nn, kk > 0);
+                mma_commit(&bars->dq_full);
+#pragma unroll
                 for (int kk = 0; kk < 8; ++kk)   // dK += dS^T Q: A = dS^T tile (keys x queries, K-major), B = Q MN-major
                     mma_ss(tmem_base + kColDK, dDS_k + desc_step_k_major(kk, kFBox), dQ_mn + kk * kDescStepMn, idesc_kn,
                            (n > 0) || (kk > 0));
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)   // dQ^T = K^T dS^T: both operands read "transposed" (MN-major)
-                    mma_ss(tP2, dK_mn + kk * kDescStepMn, dDS_mn + kk * kDescStepMn, idesc_nn, kk > 0);
-                mma_commit(&bars->dq_full);
+                mma_commit(&bars->ds_free);
                 mma_commit(&bars->st_empty[st]);
                 if (n == total_steps - 1) mma_commit(&bars->acc_full);
             }
@@ -255,77 +276,45 @@ __global__ void __launch_bounds__(kFThreads, 1) s2a_bwd_fused_kernel(const __gri
         __syncwarp();
     } else if (warp < 4) {
         // spare warps (warp 3 owns the tensor-memory allocation)
-    } else {
-        // =========================== elementwise warps =======================================
-        // Thread (quad, hf, lane): tensor-memory lane r = 32 quad + lane (a key row for S^T and dP^T,
-        // a head-dim index for dQ^T) and columns [64 hf, +64) (queries).  Its 64 bf16 P^T values
-        // (32 packed columns) go over the first half of its own S^T columns.
+    } else if (warp < 12) {
+        // =========================== elementwise group A: P^T ================================
+        // Thread (quad, hf, lane): key row r = 32 quad + lane, queries [64 hf, +64).  Its 64 bf16
+        // P^T values (32 packed columns) go over the first half of its own S^T columns.
         const int quad = warp & 3;
         const int hf = (warp - 4) >> 2;
         const int r = quad * 32 + lane;
         const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
         const uint32_t tS = t_row + kColS + hf * 64;
-        const uint32_t tP2 = t_row + kColP2 + hf * 64;
         const float c2 = p.scale_log2;
         const uint64_t c2x2 = f2_pack(c2, c2), nl2e = f2_pack(-kLog2eF, -kLog2eF);
-        auto lds4 = [](uint32_t a) {
-            float4 v;
-            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a));
-            return v;
-        };
-        // add this thread's 64 columns of dQ^T (head-dim index r, queries 64 hf ..) to the fp32
-        // accumulator of the step's query tile, then hand the columns back
-        auto drain_dq = [&](int hq_prev, int tq0_prev, uint32_t parity) -> bool {
-            if (!mbar_wait(&bars->dq_full, parity, ctx, kWaitBwdFused + 7)) return false;
-            tc_fence_after();
-            float* base = p.dq_acc + ((static_cast<size_t>(b) * geo.N + tq0_prev + hf * 64) * geo.H + hq_prev) * kHD + r;
-            const size_t col_stride = static_cast<size_t>(geo.H) * kHD;
-            uint32_t v0[32], v1[32];
-            tmem_ld_32x32(tP2, v0);
-            tmem_ld_32x32(tP2 + 32, v1);
-            tmem_wait_ld();
-            tc_fence_before();
-            mbar_arrive(&bars->dq_drained);
-#pragma unroll
-            for (int c = 0; c < 32; ++c)
-                asm volatile("red.global.add.f32 [%0], %1;" ::"l"(base + c * col_stride), "f"(__uint_as_float(v0[c])) : "memory");
-#pragma unroll
-            for (int c = 0; c < 32; ++c)
-                asm volatile("red.global.add.f32 [%0], %1;" ::"l"(base + (32 + c) * col_stride), "f"(__uint_as_float(v1[c]))
-                             : "memory");
-            return true;
-        };
         bool ok = true;
-        int n = 0, hq_prev = 0, tq0_prev = 0;
+        int n = 0;
         for (int hq = hq0; ok && hq < hq0 + rep; ++hq) {
             const TileWalk w = tile_walk(geo, hq, tk0);
             for (int i = w.j; i < Tg; ++i, ++n) {
                 const int st = n % kFStages;
                 const uint32_t par = n & 1;
-                const int tq0 = mod_pos_f(w.g * geo.G + i * kTile + w.s, geo.N);
-                if (n > 0 && !drain_dq(hq_prev, tq0_prev, par ^ 1)) { ok = false; break; }
-                hq_prev = hq, tq0_prev = tq0;
-                // ---- P^T ------------------------------------------------------------------------
                 if (!mbar_wait(&bars->st_full[st], (n / kFStages) & 1, ctx, kWaitBwdFused + 8)) { ok = false; break; }
                 if (!mbar_wait(&bars->s_full, par, ctx, kWaitBwdFused + 9)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t stat_sa = smem_u32(sStat + st * 2 * kTile) + hf * 256;  // lse of my 64 queries; D is 512 B further
+                const uint32_t stat_sa = smem_u32(sStat + st * 2 * kTile) + hf * 256;  // lse of my 64 queries
                 const bool diagonal = (i == w.j);   // query x of the tile sees key row r iff r <= x
-                uint32_t pk[32];                    // bf16 P^T of my 64 columns, kept for dS^T
+                uint32_t sr[2][32];
+                tmem_ld_32x32(tS, sr[0]);
+                tmem_ld_32x32(tS + 32, sr[1]);
+                tmem_wait_ld();
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
-                    uint32_t sr[32];
-                    tmem_ld_32x32(tS + c * 32, sr);
-                    tmem_wait_ld();
+                    uint32_t pk[16];
 #pragma unroll
                     for (int e4 = 0; e4 < 8; ++e4) {
-                        const float4 l = lds4(stat_sa + (c * 32 + e4 * 4) * 4);
+                        const float4 l = lds_f4(stat_sa + (c * 32 + e4 * 4) * 4);
                         const uint64_t lp[2] = {f2_pack(l.x, l.y), f2_pack(l.z, l.w)};
 #pragma unroll
                         for (int u = 0; u < 2; ++u) {
                             const int e = e4 * 4 + 2 * u;
                             float x0, x1;
-                            f2_unpack(f2_fma(f2_pack(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), c2x2,
+                            f2_unpack(f2_fma(f2_pack(__uint_as_float(sr[c][e]), __uint_as_float(sr[c][e + 1])), c2x2,
                                              f2_mul(lp[u], nl2e)),
                                       x0, x1);
                             float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
@@ -334,26 +323,50 @@ __global__ void __launch_bounds__(kFThreads, 1) s2a_bwd_fused_kernel(const __gri
                                 if (r > x) p0 = 0.f;
                                 if (r > x + 1) p1 = 0.f;
                             }
-                            pk[c * 16 + (e >> 1)] = pack_bf16(p0, p1);
+                            pk[e >> 1] = pack_bf16(p0, p1);
                         }
                     }
-                }
-                {
-                    uint32_t lo[16], hi[16];
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) lo[e] = pk[e], hi[e] = pk[16 + e];
-                    tmem_st_32x16(tS, lo);
-                    tmem_st_32x16(tS + 16, hi);
+                    tmem_st_32x16(tS + c * 16, pk);
                 }
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(&bars->p_ready);
-                // ---- dS^T -----------------------------------------------------------------------
-                if (!mbar_wait(&bars->dp_full, par, ctx, kWaitBwdFused + 10)) { ok = false; break; }
+            }
+        }
+    } else {
+        // =========================== elementwise group B: dS^T and the dQ^T drain ============
+        // Same (quad, hf, lane) geometry: lane r is a key row for P^T / dP^T and a head-dim index
+        // for dQ^T; columns [64 hf, +64) are queries.
+        const int quad = warp & 3;
+        const int hf = (warp - 12) >> 2;
+        const int r = quad * 32 + lane;
+        const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+        const uint32_t tPt = t_row + kColS + hf * 64;     // bf16 P^T written by group A (32 packed columns)
+        const uint32_t tP2 = t_row + kColP2 + hf * 64;
+        const uint32_t ds_row = smem_u32(sDS) + hf * kFBox + r * 128;
+        const size_t col_stride = static_cast<size_t>(geo.H) * kHD;
+        bool ok = true;
+        int n = 0;
+        for (int hq = hq0; ok && hq < hq0 + rep; ++hq) {
+            const TileWalk w = tile_walk(geo, hq, tk0);
+            for (int i = w.j; i < Tg; ++i, ++n) {
+                const int st = n % kFStages;
+                const uint32_t par = n & 1;
+                const int tq0 = mod_pos_f(w.g * geo.G + i * kTile + w.s, geo.N);
+                const uint32_t stat_sa = smem_u32(sStat + st * 2 * kTile) + hf * 256 + 512;  // D of my 64 queries
+                // ---- take a copy of P^T(n) ---------------------------------------------------------
+                if (!mbar_wait(&bars->p_ready, par, ctx, kWaitBwdFused + 13)) { ok = false; break; }
                 tc_fence_after();
-                // my row of the dS^T tile: box hf (queries 64 hf ..), row r, eight 16-byte chunks whose
-                // position is permuted by (r & 7) -- the layout a 128-byte-swizzle TMA box would have
-                const uint32_t ds_row = smem_u32(sDS) + hf * kFBox + r * 128;
+                uint32_t pk[32];
+                tmem_ld_32x32(tPt, pk);
+                tmem_wait_ld();
+                tc_fence_before();
+                mbar_arrive(&bars->p_taken);
+                // ---- dS^T(n) -------------------------------------------------------------------------
+                if (!mbar_wait(&bars->dp_full, par, ctx, kWaitBwdFused + 10)) { ok = false; break; }
+                // the previous step's dK / dQ^T MMAs still read the dS^T tile until they are done
+                if (n > 0 && !mbar_wait(&bars->ds_free, par ^ 1, ctx, kWaitBwdFused + 14)) { ok = false; break; }
+                tc_fence_after();
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     uint32_t pr[32];
@@ -362,7 +375,7 @@ __global__ void __launch_bounds__(kFThreads, 1) s2a_bwd_fused_kernel(const __gri
                     uint32_t dsw[16];
 #pragma unroll
                     for (int e4 = 0; e4 < 8; ++e4) {
-                        const float4 dd = lds4(stat_sa + 512 + (c * 32 + e4 * 4) * 4);
+                        const float4 dd = lds_f4(stat_sa + (c * 32 + e4 * 4) * 4);
                         const uint64_t dp2[2] = {f2_pack(dd.x, dd.y), f2_pack(dd.z, dd.w)};
 #pragma unroll
                         for (int u = 0; u < 2; ++u) {
@@ -375,6 +388,8 @@ __global__ void __launch_bounds__(kFThreads, 1) s2a_bwd_fused_kernel(const __gri
                             dsw[e >> 1] = pack_bf16(d0, d1);
                         }
                     }
+                    // my row of the dS^T tile: box hf, row r, eight 16-byte chunks whose position is permuted
+                    // by (r & 7) -- the layout a 128-byte-swizzle TMA box would have
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4) {
                         const int chunk = c * 4 + q4;  // 8 queries per chunk
@@ -386,14 +401,33 @@ __global__ void __launch_bounds__(kFThreads, 1) s2a_bwd_fused_kernel(const __gri
                 fence_proxy_async_smem();   // the MMAs read this tile through the async proxy
                 tc_fence_before();
                 mbar_arrive(&bars->ds_ready);
+                // ---- drain dQ^T(n): head-dim index r, queries 64 hf .. --------------------------------
+                if (!mbar_wait(&bars->dq_full, par, ctx, kWaitBwdFused + 7)) { ok = false; break; }
+                tc_fence_after();
+                float* base = p.dq_acc + ((static_cast<size_t>(b) * geo.N + tq0 + hf * 64) * geo.H + hq) * kHD + r;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t v[32];
+                    tmem_ld_32x32(tP2 + c * 32, v);
+                    tmem_wait_ld();
+                    if (c == 1) {   // all of my columns are in registers: the next dP^T may overwrite them
+                        tc_fence_before();
+                        mbar_arrive(&bars->dq_drained);
+                    }
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        asm volatile("red.global.add.f32 [%0], %1;" ::"l"(base + (c * 32 + e) * col_stride),
+                                     "f"(__uint_as_float(v[e]))
+                                     : "memory");
+                }
             }
         }
-        if (ok && n > 0) ok = drain_dq(hq_prev, tq0_prev, (n - 1) & 1);
+        // ---- epilogue: dV and dK (group B's 256 threads: 64 columns of each per thread) ------------
         if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdFused + 11)) {
             tc_fence_after();
             const size_t out_row = ((static_cast<size_t>(b) * geo.N + tk0 + r) * geo.Hkv + hk) * kHD + hf * 64;
 #pragma unroll
-            for (int m = 0; m < 2; ++m) {          // m = 0: dV, m = 1: dK; each thread stores 64 columns of each
+            for (int m = 0; m < 2; ++m) {          // m = 0: dV, m = 1: dK
                 const uint32_t t_acc = t_row + (m == 0 ? kColDV : kColDK) + hf * 64;
                 const float mul = (m == 0) ? 1.0f : p.scale;
                 __nv_bfloat16* dst_row = (m == 0 ? p.dv : p.dk) + out_row;

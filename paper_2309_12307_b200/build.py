@@ -8,7 +8,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libs2a.so")
-SOURCES = ["api.cu", "fwd_kernel.cu", "bwd_kernels.cu", "bwd_fused.cu"]
+SOURCES = ["api.cu", "fwd_kernel.cu", "bwd_kernels.cu"]
 HEADERS = ["s2a_params.h", "sm100_ptx.cuh", os.path.join("..", "..", "include", "s2a.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -59,8 +59,6 @@ int prepare_device(DeviceState** out) {
         if (e != cudaSuccess) return cuda_fail(e);
         e = configure_bwd();
         if (e != cudaSuccess) return cuda_fail(e);
-        e = configure_bwd_fused();
-        if (e != cudaSuccess) return cuda_fail(e);
         e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ds.status_ptr), g_status_word);
         if (e != cudaSuccess) return cuda_fail(e);
         ds.ready = true;
@@ -169,20 +167,11 @@ int s2a_fwd(const void* q, const void* k, const void* v, void* o, float* lse, in
     return s2a_fwd_ex(q, k, v, o, lse, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2, G / 2, stream);
 }
 
-namespace {
-// bytes of the D = rowsum(dO * o) block at the start of the workspace
-size_t dsum_bytes(int B, int N, int H) {
-    const size_t bytes = static_cast<size_t>(B) * H * N * sizeof(float);
-    return (bytes + 255) & ~static_cast<size_t>(255);
-}
-}  // namespace
-
 size_t s2a_bwd_workspace_bytes(int B, int N, int H, int Hkv, int d, int G) {
     if (B <= 0 || N <= 0 || H <= 0 || Hkv <= 0 || d <= 0 || G <= 0) return 0;
     if (N % G != 0 || H % Hkv != 0) return 0;
-    // head dim 128 runs the fused kernel, which accumulates dQ in fp32 behind D
-    const size_t dq_acc = (d == 128) ? static_cast<size_t>(B) * N * H * d * sizeof(float) : 0;
-    return dsum_bytes(B, N, H) + dq_acc;
+    const size_t bytes = static_cast<size_t>(B) * H * N * sizeof(float);
+    return (bytes + 255) & ~static_cast<size_t>(255);
 }
 
 namespace {
@@ -190,7 +179,7 @@ enum : unsigned { kStagePre = 1u, kStageDkDv = 2u, kStageDq = 4u, kStageAll = 7u
 
 int bwd_impl(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO, void* dq,
              void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, float scale, int n_unshifted, int shift,
-             void* workspace, size_t workspace_bytes, void* stream, unsigned stages, bool allow_fused = true) {
+             void* workspace, size_t workspace_bytes, void* stream, unsigned stages) {
     if (!q || !k || !v || !o || !lse || !dO || !dq || !dk || !dv || !workspace) return S2A_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse) || !aligned16(dO) ||
         !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
@@ -198,52 +187,13 @@ int bwd_impl(const void* q, const void* k, const void* v, const void* o, const f
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return S2A_ERR_INVALID_ARG;
     int rc = check_shape(B, N, H, Hkv, d, G, scale, n_unshifted, shift);
     if (rc != S2A_OK) return rc;
-    const bool fused = allow_fused && d == 128;
-    if (workspace_bytes < (fused ? s2a_bwd_workspace_bytes(B, N, H, Hkv, d, G) : dsum_bytes(B, N, H)))
-        return S2A_ERR_INVALID_ARG;
+    if (workspace_bytes < s2a_bwd_workspace_bytes(B, N, H, Hkv, d, G)) return S2A_ERR_INVALID_ARG;
     DeviceState* ds = nullptr;
     rc = prepare_device(&ds);
     if (rc != S2A_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const Geometry geo = make_geometry(B, N, H, Hkv, G, n_unshifted, shift);
     float* Dsum = static_cast<float*>(workspace);
-
-    if (fused) {
-        // D, then the fp32 dQ accumulator.  Stage 0: D and clearing of the accumulator; stage 1:
-        // dk, dv and the partial sums of dq; stage 2: dq = scale * accumulator, rounded to bf16.
-        float* dq_acc = reinterpret_cast<float*>(static_cast<char*>(workspace) + dsum_bytes(B, N, H));
-        const size_t n_dq = static_cast<size_t>(B) * N * H * d;
-        cudaError_t e;
-        if (stages & kStagePre) {
-            PreParams pp;
-            pp.o = static_cast<const __nv_bfloat16*>(o), pp.dO = static_cast<const __nv_bfloat16*>(dO), pp.Dsum = Dsum;
-            pp.B = B, pp.N = N, pp.H = H;
-            e = launch_bwd_preprocess(pp, d, st);
-            if (e != cudaSuccess) return cuda_fail(e);
-            e = cudaMemsetAsync(dq_acc, 0, n_dq * sizeof(float), st);
-            if (e != cudaSuccess) return cuda_fail(e);
-        }
-        if (stages & kStageDkDv) {
-            BwdFusedParams pf;
-            memset(&pf, 0, sizeof pf);
-            if ((rc = make_tmap(&pf.tm_k, k, d, Hkv, N, B, kTile)) != S2A_OK) return rc;
-            if ((rc = make_tmap(&pf.tm_v, v, d, Hkv, N, B, kTile)) != S2A_OK) return rc;
-            if ((rc = make_tmap(&pf.tm_q, q, d, H, N, B, kTile)) != S2A_OK) return rc;
-            if ((rc = make_tmap(&pf.tm_do, dO, d, H, N, B, kTile)) != S2A_OK) return rc;
-            pf.lse = lse, pf.Dsum = Dsum, pf.dq_acc = dq_acc;
-            pf.dk = static_cast<__nv_bfloat16*>(dk), pf.dv = static_cast<__nv_bfloat16*>(dv);
-            pf.status = ds->status_ptr, pf.geo = geo, pf.scale = scale, pf.scale_log2 = scale * kLog2eHost;
-            e = launch_bwd_fused(pf, st);
-            if (e != cudaSuccess) return cuda_fail(e);
-        }
-        if (stages & kStageDq) {
-            DqConvertParams pc;
-            pc.dq_acc = dq_acc, pc.dq = static_cast<__nv_bfloat16*>(dq), pc.n = static_cast<long long>(n_dq), pc.scale = scale;
-            e = launch_dq_convert(pc, st);
-            if (e != cudaSuccess) return cuda_fail(e);
-        }
-        return S2A_OK;
-    }
 
     BwdDqParams pq;
     memset(&pq, 0, sizeof pq);
@@ -389,7 +339,7 @@ int s2a_bwd_noalloc(const void* q, const void* k, const void* v, const void* o, 
     // Every row of D that the two gradient kernels read is rewritten by the first kernel of this
     // call, so nothing left in the array by an earlier call has to be cleared.
     return bwd_impl(q, k, v, o, lse, dO, dq, dk, dv, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2,
-                    G / 2, scratch, kBuiltinScratchRows * sizeof(float), stream, kStageAll, /*allow_fused=*/false);
+                    G / 2, scratch, kBuiltinScratchRows * sizeof(float), stream, kStageAll);
 }
 
 size_t s2a_bwd_noalloc_max_rows(void) { return kBuiltinScratchRows; }

@@ -16,7 +16,6 @@ enum WaitCode : int {
     kWaitFwd = 100,
     kWaitBwdDq = 200,
     kWaitBwdDkDv = 300,
-    kWaitBwdFused = 400,
 };
 
 // Geometry of the shifted grouping (Algorithm 1): common to every kernel.
@@ -69,31 +68,7 @@ struct alignas(64) BwdDkDvParams {
     float scale, scale_log2;
 };
 
-// Fused backward (head dim 128): dK, dV and the fp32 partial sums of dQ in one kernel.
-struct alignas(64) BwdFusedParams {
-    CUtensorMap tm_k, tm_v;   // box (64, 1, 128, 1): the resident key tile
-    CUtensorMap tm_q, tm_do;  // box (64, 1, 128, 1): streamed query tiles
-    const float* lse;
-    const float* Dsum;
-    float* dq_acc;            // [B, N, H, d] fp32, zero on entry; receives sum over key tiles of dS K (unscaled)
-    __nv_bfloat16* dk;
-    __nv_bfloat16* dv;
-    int* status;
-    Geometry geo;
-    float scale, scale_log2;
-};
-
-struct DqConvertParams {
-    const float* dq_acc;      // [B, N, H, d] fp32
-    __nv_bfloat16* dq;
-    long long n;              // elements
-    float scale;
-};
-
 // Enqueue one kernel each on `stream`; return the launch error, if any.
-cudaError_t launch_bwd_fused(const BwdFusedParams& p, cudaStream_t stream);
-cudaError_t launch_dq_convert(const DqConvertParams& p, cudaStream_t stream);
-cudaError_t configure_bwd_fused();
 cudaError_t launch_fwd(const FwdParams& p, int d, cudaStream_t stream);
 cudaError_t launch_bwd_preprocess(const PreParams& p, int d, cudaStream_t stream);
 cudaError_t launch_bwd_dq(const BwdDqParams& p, int d, cudaStream_t stream);

@@ -55,8 +55,7 @@ def test_version_and_status_strings(lib):
 def test_workspace_bytes(lib):
     lib.s2a_bwd_workspace_bytes.restype = ctypes.c_size_t
     f = lib.s2a_bwd_workspace_bytes
-    # head dim 128: D plus the fp32 dQ accumulator of the fused kernel; head dim 64: D only
-    assert f(1, 32768, 32, 32, 128, 8192) == 1 * 32 * 32768 * 4 + 1 * 32768 * 32 * 128 * 4
+    assert f(1, 32768, 32, 32, 128, 8192) == 1 * 32 * 32768 * 4
     assert f(1, 1024, 4, 4, 64, 256) == 4 * 1024 * 4
     assert f(1, 1000, 4, 4, 64, 256) == 0      # N % G
     assert f(1, 1024, 6, 4, 64, 256) == 0      # H % Hkv

@@ -116,15 +116,9 @@ def test_outputs_are_deterministic_and_fully_written(s2a):
         s2a.s2a_bwd(q, k, v, o, lse, dO, G, dq=dq, dk=dk, dv=dv)
         torch.cuda.synchronize()
         outs.append((o, lse, dq, dk, dv))
-    names = ("o", "lse", "dq", "dk", "dv")
-    for name, a, b in zip(names, *outs):
-        assert not torch.isnan(a).any(), name
-        if name == "dq":
-            # head dim 128: dq is summed over key tiles with fp32 reductions in global memory, whose
-            # order is not fixed; everything else is bit-reproducible
-            assert rel_l2(a.double().cpu().numpy(), b.double().cpu().numpy()) < 1e-3
-        else:
-            assert torch.equal(a, b), name
+    for a, b in zip(*outs):
+        assert not torch.isnan(a).any()
+        assert torch.equal(a, b)
 
 
 def test_guard_bands_stay_intact(s2a):

@@ -170,8 +170,9 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
     const Geometry& geo = p.geo;
 
     const int Tg = geo.tiles_per_group;
-    const int i = Tg - 1 - static_cast<int>(blockIdx.x % Tg);  // heaviest query tiles first
-    const int unit = blockIdx.x / Tg;
+    int unit, rank;
+    decode_block(blockIdx.x, geo.B * geo.H * geo.groups, Tg, &unit, &rank);
+    const int i = Tg - 1 - rank;  // heaviest query tiles first
     const int g = unit % geo.groups;
     const int h = (unit / geo.groups) % geo.H;
     const int b = unit / (geo.groups * geo.H);
@@ -427,8 +428,8 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
     // key tile: enumerate in the rolled order of the first query head of the KV head, heaviest
     // (earliest in the group) first
     const int Tg = geo.tiles_per_group;
-    const int j0 = static_cast<int>(blockIdx.x % Tg);
-    const int unit = blockIdx.x / Tg;
+    int unit, j0;
+    decode_block(blockIdx.x, geo.B * geo.Hkv * geo.groups, Tg, &unit, &j0);
     const int g0 = unit % geo.groups;
     const int hk = (unit / geo.groups) % geo.Hkv;
     const int b = unit / (geo.groups * geo.Hkv);

@@ -74,8 +74,8 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
 
     // ---- which tile: heaviest query tiles of a group first, groups of one head adjacent -------
     const int Tg = p.geo.tiles_per_group;
-    const int it = blockIdx.x % Tg;
-    const int unit = blockIdx.x / Tg;
+    int unit, it;
+    decode_block(blockIdx.x, p.geo.B * p.geo.H * p.geo.groups, Tg, &unit, &it);
     const int i = Tg - 1 - it;                 // query tile inside the group
     const int g = unit % p.geo.groups;
     const int h = (unit / p.geo.groups) % p.geo.H;

@@ -18,6 +18,22 @@ enum WaitCode : int {
     kWaitBwdDkDv = 300,
 };
 
+// Block order shared by the tensor-core kernels.  A "unit" is one (batch, head, group); it has
+// `tiles` tiles whose cost falls with their rank (rank 0 = most work).  Units are taken in chunks of
+// kUnitChunk: inside a chunk all rank-0 tiles come first, then all rank-1 tiles, and so on.  So the
+// blocks that run together belong to a few units (their streamed operands stay in L2), heavy tiles
+// start first, and the tail of the grid consists of the lightest tiles only.
+constexpr int kUnitChunk = 8;
+__host__ __device__ inline void decode_block(long long idx, int units, int tiles, int* unit, int* rank) {
+    const long long per_chunk = static_cast<long long>(kUnitChunk) * tiles;
+    const int chunk = static_cast<int>(idx / per_chunk);
+    const int within = static_cast<int>(idx % per_chunk);
+    const int first = chunk * kUnitChunk;
+    const int in_chunk = (units - first) < kUnitChunk ? (units - first) : kUnitChunk;
+    *rank = within / in_chunk;
+    *unit = first + within % in_chunk;
+}
+
 // Geometry of the shifted grouping (Algorithm 1): common to every kernel.
 struct Geometry {
     int B, N, H, Hkv, G;

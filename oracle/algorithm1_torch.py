@@ -31,20 +31,26 @@ def _roll_second_half(x: torch.Tensor, amount: int) -> torch.Tensor:
     return torch.cat([first, torch.roll(second, shifts=amount, dims=1)], dim=2)
 
 
-def _group_causal_attention(q, k, v, scale):
-    """q, k, v: [Bg, G, H, d] -> out [Bg, G, H, d], lse [Bg, H, G]; causal inside the group."""
+def _group_causal_attention(q, k, v, scale, extra_mask=None):
+    """q, k, v: [Bg, G, H, d] -> out [Bg, G, H, d], lse [Bg, H, G]; causal inside the group.
+    extra_mask [Bg, H, G, G] (True = hidden) adds to the causal mask."""
     G = q.shape[1]
     scores = torch.einsum("bxhc,byhc->bhxy", q, k) * scale
     future = torch.ones(G, G, dtype=torch.bool).triu(1)  # y > x
     scores = scores.masked_fill(future, float("-inf"))
+    if extra_mask is not None:
+        scores = scores.masked_fill(extra_mask, float("-inf"))
     lse = torch.logsumexp(scores, dim=-1)
     probs = torch.softmax(scores, dim=-1)
     out = torch.einsum("bhxy,byhc->bxhc", probs, v)
     return out, lse
 
 
-def s2_attn(q, k, v, G, scale=None):
-    """q [B,N,H,d], k/v [B,N,Hkv,d] (fp64) -> o [B,N,H,d], lse [B,H,N]."""
+def s2_attn(q, k, v, G, scale=None, leak_free=False):
+    """q [B,N,H,d], k/v [B,N,Hkv,d] (fp64) -> o [B,N,H,d], lse [B,H,N].
+    leak_free: variant 2 of Appendix B ("a small modification on the attention mask"): in the shifted
+    heads the last group, which holds the sequence's last G/2 tokens followed by its first G/2 tokens,
+    is treated as two groups, so the front tokens do not attend the tail tokens."""
     B, N, H, d = q.shape
     Hkv = k.shape[2]
     assert N % G == 0 and G % 2 == 0 and H % 2 == 0 and H % Hkv == 0
@@ -58,7 +64,15 @@ def s2_attn(q, k, v, G, scale=None):
     # step 2
     q, k, v = (x.reshape(B * (N // G), G, H, d) for x in (q, k, v))
     # step 3
-    out, lse = _group_causal_attention(q, k, v, scale)
+    extra = None
+    if leak_free:
+        n_groups = N // G
+        extra = torch.zeros(B * n_groups, H, G, G, dtype=torch.bool)
+        last = torch.arange(B) * n_groups + (n_groups - 1)      # the wrapped group of every sequence
+        # queries in the second half of that group (the front tokens) do not see its first half
+        for bg in last.tolist():
+            extra[bg, H // 2:, G // 2:, : G // 2] = True
+    out, lse = _group_causal_attention(q, k, v, scale, extra)
     # step 4
     out = _roll_second_half(out.reshape(B, N, H, d), G // 2)
     lse = lse.reshape(B, N // G, H, G).permute(0, 2, 1, 3).reshape(B, H, N)  # rolled token order
@@ -66,11 +80,11 @@ def s2_attn(q, k, v, G, scale=None):
     return out, lse.contiguous()
 
 
-def s2_attn_grads(q, k, v, dO, G, scale=None):
+def s2_attn_grads(q, k, v, dO, G, scale=None, leak_free=False):
     """Autograd gradients of sum(o * dO) w.r.t. q, k, v (all fp64)."""
     q = q.detach().clone().requires_grad_(True)
     k = k.detach().clone().requires_grad_(True)
     v = v.detach().clone().requires_grad_(True)
-    o, _ = s2_attn(q, k, v, G, scale)
+    o, _ = s2_attn(q, k, v, G, scale, leak_free)
     (o * dO).sum().backward()
     return q.grad, k.grad, v.grad

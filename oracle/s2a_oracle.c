@@ -67,6 +67,7 @@ typedef struct {
     int shift;       /* G/2 in the paper; sign = roll direction                 */
     int dtype;
     double scale;
+    int leak_free;   /* variant 2 of Appendix B: the wrapped tokens form a group of their own */
 } s2a_dims;
 
 static double bf16_to_f64(uint16_t bits) {
@@ -95,6 +96,35 @@ static int mod_n(long long x, int n) {
 /* shift of head h (Section 3.2: half of the heads use the shifted partition) */
 static int head_shift(const s2a_dims* D, int h) { return h < D->n_unshifted ? 0 : D->shift; }
 
+/*
+ * Variant 2 (Appendix B, "uses individual groups for the shifted tokens"): in a shifted head the
+ * group that wraps around the sequence end -- it holds the last tokens of the sequence followed by
+ * the first ones -- is cut in two at the wrap, so the front tokens no longer see the tail tokens.
+ * pw is the rolled position of original token 0; the cut applies to the group containing it
+ * (unless pw is a group boundary, where there is nothing to cut).
+ */
+static int wrap_pos(const s2a_dims* D, int s) { return mod_n(-(long long)s, D->N); }
+
+/* first rolled position attended by the query at rolled position p (head with shift s) */
+static int first_attended(const s2a_dims* D, int s, int p) {
+    const int g_first = (p / D->G) * D->G;
+    if (D->leak_free && s != 0) {
+        const int pw = wrap_pos(D, s);
+        if (pw > g_first && pw <= p) return pw;
+    }
+    return g_first;
+}
+
+/* one past the last rolled position whose query attends the key at rolled position pk */
+static int end_attending(const s2a_dims* D, int s, int pk) {
+    const int g_end = (pk / D->G + 1) * D->G;
+    if (D->leak_free && s != 0) {
+        const int pw = wrap_pos(D, s);
+        if (pw > pk && pw < g_end) return pw;
+    }
+    return g_end;
+}
+
 static size_t q_off(const s2a_dims* D, int b, int t, int h) {
     return (((size_t)b * D->N + t) * D->H + h) * (size_t)D->d;
 }
@@ -117,8 +147,7 @@ static double fwd_row(const s2a_dims* D, const void* q, const void* k, const voi
     const int s = head_shift(D, h);
     const int hk = h / (D->H / D->Hkv);
     const int p = mod_n((long long)t - s, D->N);
-    const int g = p / D->G;
-    const int p_first = g * D->G;
+    const int p_first = first_attended(D, s, p);
     const int n_att = p - p_first + 1;
 
     load_row(q, q_off(D, b, t, h), D->d, D->dtype, qrow);
@@ -158,9 +187,9 @@ static int check_dims(const s2a_dims* D) {
  * rows != NULL: n_rows triples (b,h,t); o is [n_rows,d], lse is [n_rows].
  */
 int s2a_oracle_fwd_ex(const void* q, const void* k, const void* v, int dtype, int B, int N, int H, int Hkv, int d,
-                      int G, double scale, int n_unshifted, int shift, const int* rows, long long n_rows,
-                      double* o, double* lse) {
-    s2a_dims D = {B, N, H, Hkv, d, G, n_unshifted, shift, dtype, scale};
+                      int G, double scale, int n_unshifted, int shift, int leak_free, const int* rows,
+                      long long n_rows, double* o, double* lse) {
+    s2a_dims D = {B, N, H, Hkv, d, G, n_unshifted, shift, dtype, scale, leak_free};
     if (check_dims(&D)) return -1;
     const long long total = rows ? n_rows : (long long)B * H * N;
     int err = 0;
@@ -198,7 +227,7 @@ int s2a_oracle_fwd_ex(const void* q, const void* k, const void* v, int dtype, in
 int s2a_oracle_fwd(const void* q, const void* k, const void* v, int dtype, int B, int N, int H, int Hkv, int d,
                    int G, double scale, const int* rows, long long n_rows, double* o, double* lse) {
     if ((G & 1) || (H & 1)) return -1;
-    return s2a_oracle_fwd_ex(q, k, v, dtype, B, N, H, Hkv, d, G, scale, H / 2, G / 2, rows, n_rows, o, lse);
+    return s2a_oracle_fwd_ex(q, k, v, dtype, B, N, H, Hkv, d, G, scale, H / 2, G / 2, 0, rows, n_rows, o, lse);
 }
 
 /*
@@ -211,9 +240,10 @@ int s2a_oracle_fwd(const void* q, const void* k, const void* v, int dtype, int B
  * summed on its own from the definition.
  */
 int s2a_oracle_bwd_ex(const void* q, const void* k, const void* v, const void* dO, int dtype, int B, int N, int H,
-                      int Hkv, int d, int G, double scale, int n_unshifted, int shift, const int* q_rows,
-                      long long n_q, const int* kv_rows, long long n_kv, double* dq, double* dk, double* dv) {
-    s2a_dims D = {B, N, H, Hkv, d, G, n_unshifted, shift, dtype, scale};
+                      int Hkv, int d, int G, double scale, int n_unshifted, int shift, int leak_free,
+                      const int* q_rows, long long n_q, const int* kv_rows, long long n_kv, double* dq, double* dk,
+                      double* dv) {
+    s2a_dims D = {B, N, H, Hkv, d, G, n_unshifted, shift, dtype, scale, leak_free};
     if (check_dims(&D)) return -1;
     const int r = H / Hkv;
     const size_t n_stat = (size_t)B * H * N;
@@ -242,7 +272,7 @@ int s2a_oracle_bwd_ex(const void* q, const void* k, const void* v, const void* d
             for (int h = hk * r; h < (hk + 1) * r; ++h) {
                 const int s = head_shift(&D, h);
                 const int pk = mod_n((long long)tk - s, N);
-                const int g_end = (pk / G + 1) * G; /* queries at rolled positions pk .. g_end-1 attend tk */
+                const int g_end = end_attending(&D, s, pk); /* queries at rolled positions pk .. g_end-1 attend tk */
                 for (int p = pk; p < g_end; ++p) need[((size_t)b * H + h) * N + mod_n((long long)p + s, N)] = 1;
             }
         }
@@ -290,7 +320,7 @@ int s2a_oracle_bwd_ex(const void* q, const void* k, const void* v, const void* d
                 const int s = head_shift(&D, h);
                 const int hk = h / r;
                 const int p = mod_n((long long)t - s, N);
-                const int p_first = (p / G) * G;
+                const int p_first = first_attended(&D, s, p);
                 double* out = q_rows ? dq + (size_t)i * d : dq + q_off(&D, b, t, h);
                 for (int c = 0; c < d; ++c) out[c] = 0.0;
                 load_row(q, q_off(&D, b, t, h), d, dtype, qrow);
@@ -324,7 +354,7 @@ int s2a_oracle_bwd_ex(const void* q, const void* k, const void* v, const void* d
                 for (int h = hk * r; h < (hk + 1) * r; ++h) {
                     const int s = head_shift(&D, h);
                     const int pk = mod_n((long long)tk - s, N);
-                    const int g_end = (pk / G + 1) * G;
+                    const int g_end = end_attending(&D, s, pk);
                     for (int p = pk; p < g_end; ++p) {
                         const int t = mod_n((long long)p + s, N);
                         const size_t si = ((size_t)b * H + h) * N + t;
@@ -350,7 +380,7 @@ int s2a_oracle_bwd(const void* q, const void* k, const void* v, const void* dO, 
                    int Hkv, int d, int G, double scale, const int* q_rows, long long n_q, const int* kv_rows,
                    long long n_kv, double* dq, double* dk, double* dv) {
     if ((G & 1) || (H & 1)) return -1;
-    return s2a_oracle_bwd_ex(q, k, v, dO, dtype, B, N, H, Hkv, d, G, scale, H / 2, G / 2, q_rows, n_q, kv_rows,
+    return s2a_oracle_bwd_ex(q, k, v, dO, dtype, B, N, H, Hkv, d, G, scale, H / 2, G / 2, 0, q_rows, n_q, kv_rows,
                              n_kv, dq, dk, dv);
 }
 

@@ -37,9 +37,9 @@ def _load():
         build()
         lib = ctypes.CDLL(_LIB)
         P, I, LL, D = ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong, ctypes.c_double
-        lib.s2a_oracle_fwd_ex.argtypes = [P, P, P, I, I, I, I, I, I, I, D, I, I, P, LL, P, P]
+        lib.s2a_oracle_fwd_ex.argtypes = [P, P, P, I, I, I, I, I, I, I, D, I, I, I, P, LL, P, P]
         lib.s2a_oracle_fwd_ex.restype = I
-        lib.s2a_oracle_bwd_ex.argtypes = [P, P, P, P, I, I, I, I, I, I, I, D, I, I, P, LL, P, LL, P, P, P]
+        lib.s2a_oracle_bwd_ex.argtypes = [P, P, P, P, I, I, I, I, I, I, I, D, I, I, I, P, LL, P, LL, P, P, P]
         lib.s2a_oracle_bwd_ex.restype = I
         lib.s2a_oracle_attended.argtypes = [I, I, I, I, I, P]
         lib.s2a_oracle_attended.restype = I
@@ -90,8 +90,9 @@ def _defaults(H, G, d, scale, n_unshifted, shift):
     return float(scale), int(n_unshifted), int(shift)
 
 
-def fwd(q, k, v, G, scale=None, rows=None, n_unshifted=None, shift=None):
-    """o, lse.  rows=None: o [B,N,H,d], lse [B,H,N].  rows=[(b,h,t),...]: o [n,d], lse [n]."""
+def fwd(q, k, v, G, scale=None, rows=None, n_unshifted=None, shift=None, leak_free=False):
+    """o, lse.  rows=None: o [B,N,H,d], lse [B,H,N].  rows=[(b,h,t),...]: o [n,d], lse [n].
+    leak_free=True is variant 2 of Appendix B: the wrapped group of a shifted head is cut at the wrap."""
     B, N, H, d = q.shape
     Hkv = k.shape[2]
     scale, n_unshifted, shift = _defaults(H, G, d, scale, n_unshifted, shift)
@@ -106,14 +107,14 @@ def fwd(q, k, v, G, scale=None, rows=None, n_unshifted=None, shift=None):
     else:
         o = np.empty((n, d), dtype=np.float64)
         lse = np.empty((n,), dtype=np.float64)
-    rc = _load().s2a_oracle_fwd_ex(qp, kp, vp, dt, B, N, H, Hkv, d, G, scale, n_unshifted, shift, rp, n,
+    rc = _load().s2a_oracle_fwd_ex(qp, kp, vp, dt, B, N, H, Hkv, d, G, scale, n_unshifted, shift, int(leak_free), rp, n,
                                    o.ctypes.data, lse.ctypes.data)
     if rc:
         raise ValueError(f"s2a_oracle_fwd_ex failed ({rc})")
     return o, lse
 
 
-def bwd(q, k, v, dO, G, scale=None, q_rows=None, kv_rows=None, n_unshifted=None, shift=None):
+def bwd(q, k, v, dO, G, scale=None, q_rows=None, kv_rows=None, n_unshifted=None, shift=None, leak_free=False):
     """dq, dk, dv.  With row lists: dq [n_q,d] for (b,h,t) rows, dk/dv [n_kv,d] for (b,hkv,t) rows."""
     B, N, H, d = q.shape
     Hkv = k.shape[2]
@@ -134,7 +135,8 @@ def bwd(q, k, v, dO, G, scale=None, q_rows=None, kv_rows=None, n_unshifted=None,
         qrp = dummy.ctypes.data
     if kv_rows is not None and nkv == 0:
         krp = dummy.ctypes.data
-    rc = _load().s2a_oracle_bwd_ex(qp, kp, vp, dp, dt, B, N, H, Hkv, d, G, scale, n_unshifted, shift, qrp, nq,
+    rc = _load().s2a_oracle_bwd_ex(qp, kp, vp, dp, dt, B, N, H, Hkv, d, G, scale, n_unshifted, shift, int(leak_free),
+                                   qrp, nq,
                                    krp, nkv, dq.ctypes.data, dk.ctypes.data, dv.ctypes.data)
     if rc:
         raise ValueError(f"s2a_oracle_bwd_ex failed ({rc})")

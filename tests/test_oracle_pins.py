@@ -388,3 +388,58 @@ def test_flop_accounting_matches_papers_table():
     # and the count equals the sizes of the attended sets
     N, G, H = 32, 8, 4
     assert sum(len(orc.attended(N, H, G, h, t)) for h in range(H) for t in range(N)) == H * (N // G) * G * (G + 1) // 2
+
+
+# --------------------------------------------------------------------------- variant 2 (Appendix B)
+@pytest.mark.parametrize("B,N,G,H,Hkv,d", [(1, 16, 8, 2, 2, 4), (2, 32, 8, 4, 2, 5), (1, 16, 16, 2, 1, 4)])
+def test_leak_free_variant_equals_masked_transcription(B, N, G, H, Hkv, d):
+    """Variant 2: the wrapped group of the shifted heads is cut at the wrap.  Index form against the
+    Algorithm-1 transcription with the extra mask, forward and autograd backward."""
+    q, k, v, dO = make_inputs_f64(B, N, H, Hkv, d, seed=31)
+    o_ref, lse_ref = alg1.s2_attn(q, k, v, G, leak_free=True)
+    dq_ref, dk_ref, dv_ref = alg1.s2_attn_grads(q, k, v, dO, G, leak_free=True)
+    o, lse = orc.fwd(q, k, v, G, leak_free=True)
+    dq, dk, dv = orc.bwd(q, k, v, dO, G, leak_free=True)
+    np.testing.assert_allclose(o, o_ref.numpy(), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(lse, lse_ref.numpy(), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(dq, dq_ref.numpy(), rtol=0, atol=1e-11)
+    np.testing.assert_allclose(dk, dk_ref.numpy(), rtol=0, atol=1e-11)
+    np.testing.assert_allclose(dv, dv_ref.numpy(), rtol=0, atol=1e-11)
+
+
+def test_leak_free_variant_removes_exactly_the_leak():
+    """With variant 2 the first G/2 tokens of a shifted head are plain causal attention over
+    themselves, the last G/2 tokens likewise, and every other row equals the default method."""
+    B, N, G, H, Hkv, d = 1, 64, 16, 4, 4, 8
+    q, k, v, dO = make_inputs_f64(B, N, H, Hkv, d, seed=37)
+    o_def, _ = orc.fwd(q, k, v, G)
+    o_v2, lse_v2 = orc.fwd(q, k, v, G, leak_free=True)
+    half = G // 2
+    for h in range(H // 2, H):
+        for sl in (slice(0, half), slice(N - half, N)):
+            o_ref, lse_ref = _full_causal_attention(q[0, sl, h], k[0, sl, h], v[0, sl, h], 1 / math.sqrt(d))
+            np.testing.assert_allclose(o_v2[0, sl, h], o_ref.numpy(), atol=1e-12)
+            np.testing.assert_allclose(lse_v2[0, h, sl], lse_ref.numpy(), atol=1e-12)
+    # only the front tokens of the shifted heads change
+    changed = np.abs(o_v2 - o_def).max(axis=-1)[0] > 1e-12     # [N, H]
+    assert not changed[:, : H // 2].any()
+    assert not changed[half:, H // 2:].any()
+    assert changed[:half, H // 2:].all()
+    # and they no longer depend on the tail tokens
+    k2, v2 = k.clone(), v.clone()
+    k2[0, N - 3] += 1.0
+    v2[0, N - 3] -= 1.0
+    o_pert, _ = orc.fwd(q, k2, v2, G, leak_free=True)
+    assert np.abs(o_pert - o_v2)[0, :half].max() == 0.0
+    # gradients: finite differences on one coordinate of each input
+    dq, dk, dv = orc.bwd(q, k, v, dO, G, leak_free=True)
+    eps = 1e-6
+    for x, grad, idx in ((q, dq, (0, 2, 3, 1)), (k, dk, (0, N - 2, 3, 0)), (v, dv, (0, 1, 2, 5))):
+        xp, xm = x.clone(), x.clone()
+        xp[idx] += eps
+        xm[idx] -= eps
+        args_p = [xp if t is x else t for t in (q, k, v)]
+        args_m = [xm if t is x else t for t in (q, k, v)]
+        lp = (orc.fwd(*args_p, G, leak_free=True)[0] * dO.numpy()).sum()
+        lm = (orc.fwd(*args_m, G, leak_free=True)[0] * dO.numpy()).sum()
+        assert abs((lp - lm) / (2 * eps) - grad[idx]) < 1e-6

@@ -76,20 +76,24 @@ int s2a_bwd(const void* q, const void* k, const void* v, const void* o, const fl
 size_t s2a_bwd_workspace_bytes(int B, int N, int H, int Hkv, int d, int G);
 
 /*
- * Generalised forms (Section 3.2 pilot study, Table 6 and Appendix B variant 1): the first
+ * Generalised forms (Section 3.2 pilot study, Table 6 and Appendix B variants 1 and 2): the first
  * `n_unshifted` heads use the unshifted partition, the remaining heads are rolled by -shift
  * tokens (shift a multiple of 128, |shift| < N; the paper's method is n_unshifted = H/2,
  * shift = G/2).  n_unshifted = H gives "pattern 1 only"; with G = N as well it is ordinary full
  * causal attention, which the fine-tuned model uses at inference.  `scale` multiplies the scores
  * (pass 1/sqrt(d) for the standard choice).  H may be odd here.
+ * flags: S2A_FLAG_LEAK_FREE selects variant 2 of Appendix B ("individual groups for the shifted
+ * tokens"): in a shifted head the group that wraps around the sequence end is cut in two at the
+ * wrap, so the sequence's first tokens no longer attend its last tokens.  Other bits must be 0.
  */
+#define S2A_FLAG_LEAK_FREE 1u
 int s2a_fwd_ex(const void* q, const void* k, const void* v, void* o, float* lse,
                int B, int N, int H, int Hkv, int d, int G,
-               float scale, int n_unshifted, int shift, void* stream);
+               float scale, int n_unshifted, int shift, unsigned flags, void* stream);
 int s2a_bwd_ex(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO,
                void* dq, void* dk, void* dv,
                int B, int N, int H, int Hkv, int d, int G,
-               float scale, int n_unshifted, int shift,
+               float scale, int n_unshifted, int shift, unsigned flags,
                void* workspace, size_t workspace_bytes, void* stream);
 
 /*

@@ -51,9 +51,9 @@ def load() -> ctypes.CDLL:
     lib.s2a_fwd.restype = I
     lib.s2a_bwd.argtypes = [P, P, P, P, P, P, P, P, P, I, I, I, I, I, I, P, Z, P]
     lib.s2a_bwd.restype = I
-    lib.s2a_fwd_ex.argtypes = [P, P, P, P, P, I, I, I, I, I, I, F, I, I, P]
+    lib.s2a_fwd_ex.argtypes = [P, P, P, P, P, I, I, I, I, I, I, F, I, I, ctypes.c_uint, P]
     lib.s2a_fwd_ex.restype = I
-    lib.s2a_bwd_ex.argtypes = [P, P, P, P, P, P, P, P, P, I, I, I, I, I, I, F, I, I, P, Z, P]
+    lib.s2a_bwd_ex.argtypes = [P, P, P, P, P, P, P, P, P, I, I, I, I, I, I, F, I, I, ctypes.c_uint, P, Z, P]
     lib.s2a_bwd_ex.restype = I
     lib.s2a_bwd_stage.argtypes = [P, P, P, P, P, P, P, P, P, I, I, I, I, I, I, P, Z, I, P]
     lib.s2a_bwd_stage.restype = I
@@ -175,8 +175,12 @@ def s2a_bwd_stage(q, k, v, o, lse, dO, G, dq, dk, dv, workspace, stage, stream=N
     _check(rc, "s2a_bwd_stage")
 
 
-def s2a_fwd_ex(q, k, v, G, scale=None, n_unshifted=None, shift=None, o=None, lse=None, stream=None):
-    """Generalised forward: heads [0, n_unshifted) unshifted, the rest rolled by -shift tokens."""
+S2A_FLAG_LEAK_FREE = 1
+
+
+def s2a_fwd_ex(q, k, v, G, scale=None, n_unshifted=None, shift=None, leak_free=False, o=None, lse=None, stream=None):
+    """Generalised forward: heads [0, n_unshifted) unshifted, the rest rolled by -shift tokens;
+    leak_free=True cuts the wrapped group of the shifted heads at the wrap (Appendix B, variant 2)."""
     B, N, H, Hkv, d = _dims(q, k)
     scale = 1.0 / math.sqrt(d) if scale is None else scale
     n_unshifted = H // 2 if n_unshifted is None else n_unshifted
@@ -184,12 +188,13 @@ def s2a_fwd_ex(q, k, v, G, scale=None, n_unshifted=None, shift=None, o=None, lse
     o = torch.empty_like(q) if o is None else o
     lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if lse is None else lse
     rc = load().s2a_fwd_ex(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), B, N, H, Hkv, d, G,
-                           scale, n_unshifted, shift, _stream_ptr(stream))
+                           scale, n_unshifted, shift, S2A_FLAG_LEAK_FREE if leak_free else 0, _stream_ptr(stream))
     _check(rc, "s2a_fwd_ex")
     return o, lse
 
 
-def s2a_bwd_ex(q, k, v, o, lse, dO, G, scale=None, n_unshifted=None, shift=None, workspace=None, stream=None):
+def s2a_bwd_ex(q, k, v, o, lse, dO, G, scale=None, n_unshifted=None, shift=None, leak_free=False, workspace=None,
+               stream=None):
     B, N, H, Hkv, d = _dims(q, k)
     scale = 1.0 / math.sqrt(d) if scale is None else scale
     n_unshifted = H // 2 if n_unshifted is None else n_unshifted
@@ -200,7 +205,7 @@ def s2a_bwd_ex(q, k, v, o, lse, dO, G, scale=None, n_unshifted=None, shift=None,
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
     rc = load().s2a_bwd_ex(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), dO.data_ptr(),
                            dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, N, H, Hkv, d, G, scale, n_unshifted, shift,
-                           workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+                           S2A_FLAG_LEAK_FREE if leak_free else 0, workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     _check(rc, "s2a_bwd_ex")
     return dq, dk, dv
 

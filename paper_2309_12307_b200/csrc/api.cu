@@ -100,13 +100,14 @@ int check_shape(int B, int N, int H, int Hkv, int d, int G, float scale, int n_u
     return S2A_OK;
 }
 
-Geometry make_geometry(int B, int N, int H, int Hkv, int G, int n_unshifted, int shift) {
+Geometry make_geometry(int B, int N, int H, int Hkv, int G, int n_unshifted, int shift, int leak_free = 0) {
     Geometry g;
     g.B = B, g.N = N, g.H = H, g.Hkv = Hkv, g.G = G;
     g.n_unshifted = n_unshifted;
     g.shift = shift;
     g.tiles_per_group = G / kTile;
     g.groups = N / G;
+    g.leak_free = leak_free;
     return g;
 }
 
@@ -137,7 +138,8 @@ const char* s2a_status_string(int status) {
 }
 
 int s2a_fwd_ex(const void* q, const void* k, const void* v, void* o, float* lse, int B, int N, int H, int Hkv, int d,
-               int G, float scale, int n_unshifted, int shift, void* stream) {
+               int G, float scale, int n_unshifted, int shift, unsigned flags, void* stream) {
+    if (flags & ~static_cast<unsigned>(S2A_FLAG_LEAK_FREE)) return S2A_ERR_INVALID_ARG;
     if (!q || !k || !v || !o || !lse) return S2A_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return S2A_ERR_INVALID_ARG;
     int rc = check_shape(B, N, H, Hkv, d, G, scale, n_unshifted, shift);
@@ -154,7 +156,7 @@ int s2a_fwd_ex(const void* q, const void* k, const void* v, void* o, float* lse,
     p.o = static_cast<__nv_bfloat16*>(o);
     p.lse = lse;
     p.status = ds->status_ptr;
-    p.geo = make_geometry(B, N, H, Hkv, G, n_unshifted, shift);
+    p.geo = make_geometry(B, N, H, Hkv, G, n_unshifted, shift, (flags & S2A_FLAG_LEAK_FREE) ? 1 : 0);
     p.scale_log2 = scale * kLog2eHost;
     cudaError_t e = launch_fwd(p, d, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? S2A_OK : cuda_fail(e);
@@ -164,7 +166,7 @@ int s2a_fwd(const void* q, const void* k, const void* v, void* o, float* lse, in
             int G, void* stream) {
     if (d <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
     if (G % (2 * kTile) != 0) return (G > 0 && N > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
-    return s2a_fwd_ex(q, k, v, o, lse, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2, G / 2, stream);
+    return s2a_fwd_ex(q, k, v, o, lse, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2, G / 2, 0u, stream);
 }
 
 size_t s2a_bwd_workspace_bytes(int B, int N, int H, int Hkv, int d, int G) {
@@ -179,7 +181,7 @@ enum : unsigned { kStagePre = 1u, kStageDkDv = 2u, kStageDq = 4u, kStageAll = 7u
 
 int bwd_impl(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO, void* dq,
              void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, float scale, int n_unshifted, int shift,
-             void* workspace, size_t workspace_bytes, void* stream, unsigned stages) {
+             void* workspace, size_t workspace_bytes, void* stream, unsigned stages, unsigned flags = 0u) {
     if (!q || !k || !v || !o || !lse || !dO || !dq || !dk || !dv || !workspace) return S2A_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse) || !aligned16(dO) ||
         !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
@@ -192,7 +194,8 @@ int bwd_impl(const void* q, const void* k, const void* v, const void* o, const f
     rc = prepare_device(&ds);
     if (rc != S2A_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const Geometry geo = make_geometry(B, N, H, Hkv, G, n_unshifted, shift);
+    if (flags & ~static_cast<unsigned>(S2A_FLAG_LEAK_FREE)) return S2A_ERR_INVALID_ARG;
+    const Geometry geo = make_geometry(B, N, H, Hkv, G, n_unshifted, shift, (flags & S2A_FLAG_LEAK_FREE) ? 1 : 0);
     float* Dsum = static_cast<float*>(workspace);
 
     BwdDqParams pq;
@@ -237,9 +240,9 @@ int bwd_impl(const void* q, const void* k, const void* v, const void* o, const f
 
 int s2a_bwd_ex(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO, void* dq,
                void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, float scale, int n_unshifted,
-               int shift, void* workspace, size_t workspace_bytes, void* stream) {
+               int shift, unsigned flags, void* workspace, size_t workspace_bytes, void* stream) {
     return bwd_impl(q, k, v, o, lse, dO, dq, dk, dv, B, N, H, Hkv, d, G, scale, n_unshifted, shift, workspace,
-                    workspace_bytes, stream, kStageAll);
+                    workspace_bytes, stream, kStageAll, flags);
 }
 
 int s2a_bwd_stage(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO,
@@ -258,7 +261,7 @@ int s2a_bwd(const void* q, const void* k, const void* v, const void* o, const fl
     if (d <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
     if (G % (2 * kTile) != 0) return (G > 0 && N > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
     return s2a_bwd_ex(q, k, v, o, lse, dO, dq, dk, dv, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2,
-                      G / 2, workspace, workspace_bytes, stream);
+                      G / 2, 0u, workspace, workspace_bytes, stream);
 }
 
 int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const void* h_dO, void* h_o, float* h_lse,

@@ -178,7 +178,8 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
     const int b = unit / (geo.groups * geo.H);
     const int hk = h / (geo.H / geo.Hkv);
     const int s = (h < geo.n_unshifted) ? 0 : geo.shift;
-    const int n_steps = 2 * (i + 1);  // key sub-tiles 0 .. 2i+1 of the group
+    const int n_begin = 2 * first_key_tile(geo, s, g, i);
+    const int n_steps = 2 * (i + 1) - n_begin;  // key sub-tiles n_begin .. 2i+1 of the group (n_begin = 0 by default)
     const int tq0 = mod_pos(g * geo.G + i * kTile + s, geo.N);
 
     if (threadIdx.x == 0) {
@@ -224,7 +225,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
             for (; n < n_steps; ++n) {
                 const int st = n % C::kStages;
                 const uint32_t ph = (n / C::kStages) & 1;
-                const int tk0 = mod_pos(g * geo.G + n * kSubTile + s, geo.N);
+                const int tk0 = mod_pos(g * geo.G + (n_begin + n) * kSubTile + s, geo.N);
                 if (!mbar_wait(&bars->st_empty[st], ph ^ 1, ctx, kWaitBwdDq + 1)) break;
                 mbar_expect_tx(&bars->st_full[st], C::kStageBytes);
                 uint8_t* sK = sStage + st * C::kStageBytes;
@@ -332,10 +333,10 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
             tmem_ld_32x32(tP, pr);
             tmem_wait_ld();
             uint32_t pk[16];
-            if (n >= 2 * i) {
-                // diagonal sub-tiles: key x is visible to query row r iff 64 n + x <= 128 i + r
+            if (n_begin + n >= 2 * i) {
+                // diagonal sub-tiles: key x of sub-tile m is visible to query row r iff 64 m + x <= 128 i + r
                 float ds[32];
-                const int lim = i * kTile + row - n * kSubTile - half * 32;  // visible iff e <= lim
+                const int lim = i * kTile + row - (n_begin + n) * kSubTile - half * 32;  // visible iff e <= lim
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
                     float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, neg_lse2));
@@ -397,7 +398,7 @@ __device__ __forceinline__ HeadWalk head_walk(const Geometry& geo, int hq, int t
     w.g = pos / geo.G;
     w.j = (pos % geo.G) / kTile;
     w.n_begin = 2 * w.j;
-    w.n_end = 2 * geo.tiles_per_group;
+    w.n_end = 2 * end_query_tile(geo, w.s, w.g, w.j);
     return w;
 }
 

@@ -82,7 +82,8 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
     const int b = unit / (p.geo.groups * p.geo.H);
     const int hk = h / (p.geo.H / p.geo.Hkv);
     const int s = (h < p.geo.n_unshifted) ? 0 : p.geo.shift;
-    const int n_kv = i + 1;                    // causal: key tiles 0..i of the same group
+    const int j_begin = first_key_tile(p.geo, s, g, i);
+    const int n_kv = i + 1 - j_begin;          // causal: key tiles j_begin..i of the same group (j_begin = 0 by default)
     // original token of rolled position x:  (x + s) mod N
     auto orig_token = [&](int rolled) {
         int t = (rolled + s) % p.geo.N;
@@ -131,7 +132,7 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
             for (; j < n_kv; ++j) {
                 const int st = j % C::kStages;
                 const uint32_t ph = (j / C::kStages) & 1;
-                const int tk0 = orig_token(g * p.geo.G + j * kTile);
+                const int tk0 = orig_token(g * p.geo.G + (j_begin + j) * kTile);
                 if (!mbar_wait(k_empty + st, ph ^ 1, ctx, kWaitFwd + 1)) break;
                 mbar_expect_tx(k_full + st, C::kTileBytes);
                 for (int bx = 0; bx < C::kBoxes; ++bx)
@@ -249,7 +250,7 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
             tc_fence_after();
             // pass 1: row maximum of this thread's 64 columns (the scores are read again in pass 2,
             // 32 at a time, which keeps the register footprint small enough for two CTAs per SM)
-            const bool diagonal = (j == i);    // key x of the tile is visible to query row r iff x <= r
+            const bool diagonal = (j == n_kv - 1);    // key x of the tile is visible to query row r iff x <= r
             const int lim = row - half * 64;   // visible iff (column within this half) <= lim
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll

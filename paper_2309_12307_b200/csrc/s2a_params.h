@@ -41,7 +41,31 @@ struct Geometry {
     int shift;            // tokens; the rest of the heads are rolled by -shift (G/2 in Algorithm 1)
     int tiles_per_group;  // G / 128
     int groups;           // N / G
+    int leak_free;        // variant 2 of Appendix B: cut the wrapped group of a shifted head at the wrap
 };
+
+// Variant 2: in a head with shift s != 0 the group that contains the rolled position of original
+// token 0 (pw = -s mod N) is cut in two there; queries at or after the cut attend keys from the cut
+// on, keys before the cut are attended by queries before the cut only.  Both in units of 128-token
+// tiles inside the group; without the variant they are 0 and tiles_per_group.
+__host__ __device__ inline int first_key_tile(const Geometry& geo, int s, int g, int i) {
+    if (geo.leak_free && s != 0) {
+        int pw = (-s) % geo.N;
+        if (pw < 0) pw += geo.N;
+        const int iw = (pw % geo.G) / kTile;
+        if (g == pw / geo.G && iw > 0 && i >= iw) return iw;
+    }
+    return 0;
+}
+__host__ __device__ inline int end_query_tile(const Geometry& geo, int s, int g, int j) {
+    if (geo.leak_free && s != 0) {
+        int pw = (-s) % geo.N;
+        if (pw < 0) pw += geo.N;
+        const int iw = (pw % geo.G) / kTile;
+        if (g == pw / geo.G && iw > 0 && j < iw) return iw;
+    }
+    return geo.tiles_per_group;
+}
 
 struct alignas(64) FwdParams {
     CUtensorMap tm_q;  // bf16 (d, H,   N, B), box (64, 1, 128, 1), 128-byte swizzle

@@ -89,6 +89,9 @@ def test_generalised_shift_and_head_split(s2a):
         dict(n_unshifted=0, shift=G // 2),
         dict(n_unshifted=1, shift=128, scale=0.2),
         dict(n_unshifted=2, shift=-(G // 2)),
+        dict(leak_free=True),                               # Appendix B, variant 2
+        dict(n_unshifted=1, shift=128, leak_free=True),
+        dict(n_unshifted=2, shift=-(G // 2), leak_free=True),
     ]
     for ex in cases:
         o, lse, dq, dk, dv = run_gpu(s2a, q, k, v, dO, G, **ex)
@@ -102,6 +105,25 @@ def test_generalised_shift_and_head_split(s2a):
     o, lse, dq, dk, dv = run_gpu(s2a, q, k, v, dO, N, n_unshifted=H, shift=0)
     o_ref, _ = orc.fwd(q, k, v, N, n_unshifted=H, shift=0)
     assert np.abs(o - o_ref).max() <= O_ATOL
+
+
+def test_leak_free_variant_matches_oracle(s2a):
+    """Appendix B, variant 2 on a head-dim-128 GQA shape with eight tiles per group: the wrapped group
+    of the shifted heads is cut at the wrap (tile 4 of 8)."""
+    B, N, G, H, Hkv, d = 2, 2048, 1024, 4, 2, 128
+    q, k, v, dO = make_inputs(B, N, H, Hkv, d, seed=5)
+    o, lse, dq, dk, dv = run_gpu(s2a, q, k, v, dO, G, leak_free=True)
+    o_ref, lse_ref = orc.fwd(q, k, v, G, leak_free=True)
+    dq_ref, dk_ref, dv_ref = orc.bwd(q, k, v, dO, G, leak_free=True)
+    assert np.abs(o - o_ref).max() <= O_ATOL
+    assert np.abs(lse - lse_ref).max() <= LSE_ATOL
+    for got, want in ((dq, dq_ref), (dk, dk_ref), (dv, dv_ref)):
+        assert rel_l2(got, want) <= GRAD_REL_L2
+    # the variant changes only the first G/2 tokens of the shifted heads
+    o_def, _, _, _, _ = run_gpu(s2a, q, k, v, dO, G)
+    assert np.array_equal(o[:, G // 2:], o_def[:, G // 2:])
+    assert np.array_equal(o[:, :, : H // 2], o_def[:, :, : H // 2])
+    assert np.abs(o[:, : G // 2, H // 2:] - o_def[:, : G // 2, H // 2:]).max() > 1e-3
 
 
 def test_outputs_are_deterministic_and_fully_written(s2a):

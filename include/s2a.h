@@ -6,10 +6,10 @@
  *   - the N tokens of a sequence are cut into N/G groups of G consecutive tokens;
  *   - in the second half of the heads (h >= H/2) the tokens are rolled by -G/2 first, so that the
  *     group boundaries sit half a group later and the last group wraps around the sequence end
- *     (Algorithm 1, key line 1; Section 3.2: with N=8192, G=2048 the first shifted group holds
+ *     (Algorithm 1, its shift step; Section 3.2: with N=8192, G=2048 the first shifted group holds
  *     tokens 1025..3072 and the first and last 1024 tokens share a group);
  *   - causal softmax attention, scores scaled by 1/sqrt(d), runs inside each group in rolled order;
- *   - the second half of the heads is rolled back by +G/2 (key line 2), so every output is indexed
+ *   - the second half of the heads is rolled back by +G/2 (Algorithm 1, its roll-back step), so every output is indexed
  *     by ORIGINAL token position.
  * Grouped-query attention: query head h reads KV head floor(h / (H/Hkv)) at the same (rolled)
  * coordinates as itself.  The wrapped group of a shifted head is kept as the paper's default

@@ -3,4 +3,4 @@
 `inputs` (seeded synthetic tensors) is importable anywhere; `binding` loads the
 CUDA library and raises if it has not been built.
 """
-__all__ = ["inputs", "binding"]
+__all__ = ["inputs", "binding", "autograd", "replicas"]

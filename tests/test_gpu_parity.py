@@ -126,6 +126,22 @@ def test_leak_free_variant_matches_oracle(s2a):
     assert np.abs(o[:, : G // 2, H // 2:] - o_def[:, : G // 2, H // 2:]).max() > 1e-3
 
 
+def test_autograd_wrapper_matches_oracle(s2a):
+    from paper_2309_12307_b200.autograd import s2_attn
+
+    B, N, G, H, Hkv, d = 1, 1024, 512, 4, 2, 128
+    q, k, v, dO = make_inputs(B, N, H, Hkv, d, seed=6)
+    qd, kd, vd = (x.cuda().requires_grad_(True) for x in (q, k, v))
+    o = s2_attn(qd, kd, vd, G)
+    (o.float() * dO.cuda().float()).sum().backward()
+    torch.cuda.synchronize()
+    o_ref, _ = orc.fwd(q, k, v, G)
+    dq_ref, dk_ref, dv_ref = orc.bwd(q, k, v, dO, G)
+    assert np.abs(o.detach().double().cpu().numpy() - o_ref).max() <= O_ATOL
+    for got, want in ((qd.grad, dq_ref), (kd.grad, dk_ref), (vd.grad, dv_ref)):
+        assert rel_l2(got.double().cpu().numpy(), want) <= GRAD_REL_L2
+
+
 def test_outputs_are_deterministic_and_fully_written(s2a):
     B, N, G, H, Hkv, d = 1, 1024, 256, 4, 2, 128
     q, k, v, dO = (x.cuda() for x in make_inputs(B, N, H, Hkv, d, seed=2))

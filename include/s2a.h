@@ -97,6 +97,19 @@ int s2a_bwd_ex(const void* q, const void* k, const void* v, const void* o, const
                void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The calling convention of Algorithm 1 itself: queries, keys and values packed in one tensor
+ *   qkv  : bf16 [B, N, 3, H, d]   (index 0 = q, 1 = k, 2 = v; H query heads = H KV heads)
+ *   dqkv : bf16 [B, N, 3, H, d]   gradients in the same packing (overwritten)
+ * o, dO [B, N, H, d] and lse [B, H, N] stay dense.  Nothing is unpacked or copied: the packed layout
+ * only changes the strides of the TMA tensor maps and of the gradient stores.  Semantics, shape
+ * limits, workspace and errors are those of s2a_fwd / s2a_bwd with Hkv = H.
+ */
+int s2a_fwd_packed(const void* qkv, void* o, float* lse, int B, int N, int H, int d, int G, void* stream);
+int s2a_bwd_packed(const void* qkv, const void* o, const float* lse, const void* dO, void* dqkv,
+                   int B, int N, int H, int d, int G,
+                   void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * s2a_bwd for callers that have no scratch to give.  (The paper has no counterpart to this entry
  * point; it exists for integration reasons only.)
  *

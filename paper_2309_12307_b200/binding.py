@@ -24,7 +24,7 @@ S2A_ERR_TOO_LARGE = -5
 
 EXPORTS = [
     "s2a_fwd", "s2a_bwd", "s2a_bwd_workspace_bytes", "s2a_fwd_ex", "s2a_bwd_ex", "s2a_bwd_stage", "s2a_fwd_bwd_host",
-    "s2a_bwd_noalloc", "s2a_bwd_noalloc_max_rows",
+    "s2a_bwd_noalloc", "s2a_bwd_noalloc_max_rows", "s2a_fwd_packed", "s2a_bwd_packed",
     "s2a_device_status", "s2a_status_string", "s2a_last_cuda_error", "s2a_version",
 ]
 
@@ -60,6 +60,10 @@ def load() -> ctypes.CDLL:
     lib.s2a_bwd_noalloc.argtypes = [P, P, P, P, P, P, P, P, P, I, I, I, I, I, I, P]
     lib.s2a_bwd_noalloc.restype = I
     lib.s2a_bwd_noalloc_max_rows.restype = Z
+    lib.s2a_fwd_packed.argtypes = [P, P, P, I, I, I, I, I, P]
+    lib.s2a_fwd_packed.restype = I
+    lib.s2a_bwd_packed.argtypes = [P, P, P, P, P, I, I, I, I, I, P, Z, P]
+    lib.s2a_bwd_packed.restype = I
     lib.s2a_bwd_workspace_bytes.argtypes = [I, I, I, I, I, I]
     lib.s2a_bwd_workspace_bytes.restype = Z
     lib.s2a_fwd_bwd_host.argtypes = [P] * 18 + [I] * 6 + [P, Z, P]
@@ -164,6 +168,32 @@ def s2a_bwd_noalloc(q, k, v, o, lse, dO, G, dq, dk, dv, stream=None):
                                 _stream_ptr(stream))
     _check(rc, "s2a_bwd_noalloc")
     return dq, dk, dv
+
+
+def s2a_fwd_packed(qkv, G, o=None, lse=None, stream=None):
+    """Forward on a packed qkv tensor [B, N, 3, H, d] (the calling convention of Algorithm 1)."""
+    B, N, three, H, d = qkv.shape
+    assert three == 3
+    _require(qkv, torch.bfloat16, "qkv")
+    o = torch.empty((B, N, H, d), dtype=torch.bfloat16, device=qkv.device) if o is None else o
+    lse = torch.empty((B, H, N), dtype=torch.float32, device=qkv.device) if lse is None else lse
+    rc = load().s2a_fwd_packed(qkv.data_ptr(), o.data_ptr(), lse.data_ptr(), B, N, H, d, G, _stream_ptr(stream))
+    _check(rc, "s2a_fwd_packed")
+    return o, lse
+
+
+def s2a_bwd_packed(qkv, o, lse, dO, G, dqkv=None, workspace=None, stream=None):
+    """Backward on a packed qkv tensor; returns dqkv [B, N, 3, H, d]."""
+    B, N, three, H, d = qkv.shape
+    assert three == 3
+    dqkv = torch.empty_like(qkv) if dqkv is None else dqkv
+    need = bwd_workspace_bytes(B, N, H, H, d, G)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=qkv.device)
+    rc = load().s2a_bwd_packed(qkv.data_ptr(), o.data_ptr(), lse.data_ptr(), dO.data_ptr(), dqkv.data_ptr(), B, N, H, d, G,
+                               workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+    _check(rc, "s2a_bwd_packed")
+    return dqkv
 
 
 def s2a_bwd_stage(q, k, v, o, lse, dO, G, dq, dk, dv, workspace, stage, stream=None):

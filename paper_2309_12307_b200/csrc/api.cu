@@ -69,9 +69,12 @@ int prepare_device(DeviceState** out) {
 
 // bf16 tensor [B, N, heads, d] viewed as (d, heads, N, B); box = 64 columns x `box_rows` tokens of
 // one head, written to shared memory with the 128-byte swizzle the MMA descriptors expect.
-int make_tmap(CUtensorMap* tm, const void* base, int d, int heads, int N, int B, int box_rows) {
+// `tok_stride` = elements between consecutive tokens (heads * d when the tensor is dense; 3 * H * d for
+// the slices of a packed [B, N, 3, H, d] tensor).
+int make_tmap(CUtensorMap* tm, const void* base, int d, int heads, int N, int B, int box_rows, long long tok_stride = 0) {
+    if (tok_stride == 0) tok_stride = static_cast<long long>(heads) * d;
     const cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)heads, (cuuint64_t)N, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {(cuuint64_t)d * 2, (cuuint64_t)heads * d * 2, (cuuint64_t)N * heads * d * 2};
+    const cuuint64_t strides[3] = {(cuuint64_t)d * 2, (cuuint64_t)tok_stride * 2, (cuuint64_t)N * tok_stride * 2};
     const cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
@@ -137,8 +140,14 @@ const char* s2a_status_string(int status) {
     }
 }
 
-int s2a_fwd_ex(const void* q, const void* k, const void* v, void* o, float* lse, int B, int N, int H, int Hkv, int d,
-               int G, float scale, int n_unshifted, int shift, unsigned flags, void* stream) {
+namespace {
+// Token strides in elements; 0 means dense ([B, N, heads, d]).
+struct TokStrides {
+    long long q = 0, kv = 0, dq = 0, dkv = 0;
+};
+
+int fwd_impl(const void* q, const void* k, const void* v, void* o, float* lse, int B, int N, int H, int Hkv, int d,
+             int G, float scale, int n_unshifted, int shift, unsigned flags, void* stream, const TokStrides& ts) {
     if (flags & ~static_cast<unsigned>(S2A_FLAG_LEAK_FREE)) return S2A_ERR_INVALID_ARG;
     if (!q || !k || !v || !o || !lse) return S2A_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return S2A_ERR_INVALID_ARG;
@@ -150,9 +159,9 @@ int s2a_fwd_ex(const void* q, const void* k, const void* v, void* o, float* lse,
 
     FwdParams p;
     memset(&p, 0, sizeof p);
-    if ((rc = make_tmap(&p.tm_q, q, d, H, N, B, kTile)) != S2A_OK) return rc;
-    if ((rc = make_tmap(&p.tm_k, k, d, Hkv, N, B, kTile)) != S2A_OK) return rc;
-    if ((rc = make_tmap(&p.tm_v, v, d, Hkv, N, B, kTile)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&p.tm_q, q, d, H, N, B, kTile, ts.q)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&p.tm_k, k, d, Hkv, N, B, kTile, ts.kv)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&p.tm_v, v, d, Hkv, N, B, kTile, ts.kv)) != S2A_OK) return rc;
     p.o = static_cast<__nv_bfloat16*>(o);
     p.lse = lse;
     p.status = ds->status_ptr;
@@ -160,6 +169,24 @@ int s2a_fwd_ex(const void* q, const void* k, const void* v, void* o, float* lse,
     p.scale_log2 = scale * kLog2eHost;
     cudaError_t e = launch_fwd(p, d, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? S2A_OK : cuda_fail(e);
+}
+}  // namespace
+
+int s2a_fwd_ex(const void* q, const void* k, const void* v, void* o, float* lse, int B, int N, int H, int Hkv, int d,
+               int G, float scale, int n_unshifted, int shift, unsigned flags, void* stream) {
+    return fwd_impl(q, k, v, o, lse, B, N, H, Hkv, d, G, scale, n_unshifted, shift, flags, stream, TokStrides());
+}
+
+int s2a_fwd_packed(const void* qkv, void* o, float* lse, int B, int N, int H, int d, int G, void* stream) {
+    if (!qkv) return S2A_ERR_INVALID_ARG;
+    if (d <= 0 || H <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
+    if (G % (2 * kTile) != 0) return (G > 0 && N > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
+    const __nv_bfloat16* base = static_cast<const __nv_bfloat16*>(qkv);
+    const long long hd = static_cast<long long>(H) * d;
+    TokStrides ts;
+    ts.q = ts.kv = 3 * hd;
+    return fwd_impl(base, base + hd, base + 2 * hd, o, lse, B, N, H, H, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2,
+                    G / 2, 0u, stream, ts);
 }
 
 int s2a_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int N, int H, int Hkv, int d,
@@ -181,7 +208,8 @@ enum : unsigned { kStagePre = 1u, kStageDkDv = 2u, kStageDq = 4u, kStageAll = 7u
 
 int bwd_impl(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO, void* dq,
              void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, float scale, int n_unshifted, int shift,
-             void* workspace, size_t workspace_bytes, void* stream, unsigned stages, unsigned flags = 0u) {
+             void* workspace, size_t workspace_bytes, void* stream, unsigned stages, unsigned flags = 0u,
+             const TokStrides& ts = TokStrides()) {
     if (!q || !k || !v || !o || !lse || !dO || !dq || !dk || !dv || !workspace) return S2A_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse) || !aligned16(dO) ||
         !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
@@ -200,19 +228,21 @@ int bwd_impl(const void* q, const void* k, const void* v, const void* o, const f
 
     BwdDqParams pq;
     memset(&pq, 0, sizeof pq);
-    if ((rc = make_tmap(&pq.tm_q, q, d, H, N, B, kTile)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pq.tm_q, q, d, H, N, B, kTile, ts.q)) != S2A_OK) return rc;
     if ((rc = make_tmap(&pq.tm_do, dO, d, H, N, B, kTile)) != S2A_OK) return rc;
-    if ((rc = make_tmap(&pq.tm_k, k, d, Hkv, N, B, kSubTile)) != S2A_OK) return rc;
-    if ((rc = make_tmap(&pq.tm_v, v, d, Hkv, N, B, kSubTile)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pq.tm_k, k, d, Hkv, N, B, kSubTile, ts.kv)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pq.tm_v, v, d, Hkv, N, B, kSubTile, ts.kv)) != S2A_OK) return rc;
+    pq.dq_tok_stride = ts.dq ? ts.dq : static_cast<long long>(H) * d;
     pq.lse = lse, pq.Dsum = Dsum, pq.dq = static_cast<__nv_bfloat16*>(dq);
     pq.status = ds->status_ptr, pq.geo = geo, pq.scale = scale, pq.scale_log2 = scale * kLog2eHost;
 
     BwdDkDvParams pk;
     memset(&pk, 0, sizeof pk);
-    if ((rc = make_tmap(&pk.tm_k, k, d, Hkv, N, B, kTile)) != S2A_OK) return rc;
-    if ((rc = make_tmap(&pk.tm_v, v, d, Hkv, N, B, kTile)) != S2A_OK) return rc;
-    if ((rc = make_tmap(&pk.tm_q, q, d, H, N, B, kSubTile)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pk.tm_k, k, d, Hkv, N, B, kTile, ts.kv)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pk.tm_v, v, d, Hkv, N, B, kTile, ts.kv)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pk.tm_q, q, d, H, N, B, kSubTile, ts.q)) != S2A_OK) return rc;
     if ((rc = make_tmap(&pk.tm_do, dO, d, H, N, B, kSubTile)) != S2A_OK) return rc;
+    pk.dkv_tok_stride = ts.dkv ? ts.dkv : static_cast<long long>(Hkv) * d;
     pk.lse = lse, pk.Dsum = Dsum;
     pk.dk = static_cast<__nv_bfloat16*>(dk), pk.dv = static_cast<__nv_bfloat16*>(dv);
     pk.status = ds->status_ptr, pk.geo = geo, pk.scale = scale, pk.scale_log2 = scale * kLog2eHost;
@@ -243,6 +273,20 @@ int s2a_bwd_ex(const void* q, const void* k, const void* v, const void* o, const
                int shift, unsigned flags, void* workspace, size_t workspace_bytes, void* stream) {
     return bwd_impl(q, k, v, o, lse, dO, dq, dk, dv, B, N, H, Hkv, d, G, scale, n_unshifted, shift, workspace,
                     workspace_bytes, stream, kStageAll, flags);
+}
+
+int s2a_bwd_packed(const void* qkv, const void* o, const float* lse, const void* dO, void* dqkv, int B, int N, int H,
+                   int d, int G, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!qkv || !dqkv) return S2A_ERR_INVALID_ARG;
+    if (d <= 0 || H <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
+    if (G % (2 * kTile) != 0) return (G > 0 && N > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
+    const __nv_bfloat16* in = static_cast<const __nv_bfloat16*>(qkv);
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(dqkv);
+    const long long hd = static_cast<long long>(H) * d;
+    TokStrides ts;
+    ts.q = ts.kv = ts.dq = ts.dkv = 3 * hd;
+    return bwd_impl(in, in + hd, in + 2 * hd, o, lse, dO, out, out + hd, out + 2 * hd, B, N, H, H, d, G,
+                    1.0f / sqrtf(static_cast<float>(d)), H / 2, G / 2, workspace, workspace_bytes, stream, kStageAll, 0u, ts);
 }
 
 int s2a_bwd_stage(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO,

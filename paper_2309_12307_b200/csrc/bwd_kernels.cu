@@ -366,7 +366,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         }
         if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDq + 6)) {
             tc_fence_after();
-            __nv_bfloat16* dst = p.dq + ((static_cast<size_t>(b) * geo.N + tq0 + row) * geo.H + h) * HD;
+            __nv_bfloat16* dst = p.dq + (static_cast<size_t>(b) * geo.N + tq0 + row) * p.dq_tok_stride + static_cast<size_t>(h) * HD;
             store_acc_cols<HD / 2>(t_row + kColAcc + half * (HD / 2), p.scale, dst + half * (HD / 2));
         }
     }
@@ -670,7 +670,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         }
         if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDkDv + 7)) {
             tc_fence_after();
-            const size_t out_row = ((static_cast<size_t>(b) * geo.N + tk0 + row) * geo.Hkv + hk) * HD;
+            const size_t out_row = (static_cast<size_t>(b) * geo.N + tk0 + row) * p.dkv_tok_stride + static_cast<size_t>(hk) * HD;
             if (half == 0) store_acc_cols<HD>(t_row + kColDV, 1.0f, p.dv + out_row);
             else store_acc_cols<HD>(t_row + kColDK, p.scale, p.dk + out_row);
         }

@@ -91,6 +91,7 @@ struct alignas(64) BwdDqParams {
     const float* lse;         // [B, H, N]
     const float* Dsum;        // [B, H, N]
     __nv_bfloat16* dq;
+    long long dq_tok_stride;  // elements between consecutive tokens of dq (H * d when dense)
     int* status;
     Geometry geo;
     float scale, scale_log2;
@@ -103,6 +104,7 @@ struct alignas(64) BwdDkDvParams {
     const float* Dsum;
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
+    long long dkv_tok_stride;  // elements between consecutive tokens of dk and dv (Hkv * d when dense)
     int* status;
     Geometry geo;
     float scale, scale_log2;

@@ -126,6 +126,22 @@ def test_leak_free_variant_matches_oracle(s2a):
     assert np.abs(o[:, : G // 2, H // 2:] - o_def[:, : G // 2, H // 2:]).max() > 1e-3
 
 
+def test_packed_qkv_equals_separate_tensors(s2a):
+    """Algorithm 1 takes qkv packed as [B, N, 3, H, d]; the packed entry points must give exactly
+    what the separate-tensor entry points give on the same values (only strides differ)."""
+    B, N, G, H, d = 2, 1024, 512, 4, 128
+    q, k, v, dO = (x.cuda() for x in make_inputs(B, N, H, H, d, seed=7))
+    qkv = torch.stack([q, k, v], dim=2).contiguous()          # [B, N, 3, H, d]
+    o, lse = s2a.s2a_fwd(q, k, v, G)
+    dq, dk, dv = s2a.s2a_bwd(q, k, v, o, lse, dO, G)
+    o_p, lse_p = s2a.s2a_fwd_packed(qkv, G)
+    dqkv = torch.full_like(qkv, float("nan"))
+    s2a.s2a_bwd_packed(qkv, o_p, lse_p, dO, G, dqkv=dqkv)
+    torch.cuda.synchronize()
+    assert torch.equal(o, o_p) and torch.equal(lse, lse_p)
+    assert torch.equal(dqkv[:, :, 0], dq) and torch.equal(dqkv[:, :, 1], dk) and torch.equal(dqkv[:, :, 2], dv)
+
+
 def test_autograd_wrapper_matches_oracle(s2a):
     from paper_2309_12307_b200.autograd import s2_attn
 

@@ -24,9 +24,15 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).  Calls only enqueue
  *     work and return without synchronising.
  *   - Return value: S2A_OK (0) or a negative s2a_status.  On error nothing was enqueued.
- *   - Supported shapes: d in {64, 128}; G a multiple of 256 (so that G/2 is a whole number of
- *     128-token tiles); N a multiple of G; H even; H a multiple of Hkv; pointers 16-byte aligned;
- *     a device of compute capability 10.x.  Anything else is rejected, never approximated.
+ *   - Supported shapes: d in {64, 128}; N a multiple of G, N >= 128; G a multiple of 8 (so that every
+ *     run of tokens of a group, shifted by G/2 or not, starts and ends on a multiple of 4 tokens);
+ *     H even; H a multiple of Hkv; pointers 16-byte aligned; a device of compute capability 10.x.
+ *     G need not be a multiple of the kernels' 128-token tile (the paper's G = N/4 of N = 100,000 is
+ *     25,000): a group is then covered by tiles whose last one is partly masked, and the group that
+ *     wraps around the end of the sequence by two such runs of tiles.  Anything else is rejected,
+ *     never approximated.
+ *   - Rows of a partly masked tile that belong to a neighbouring group are read (and masked), so a
+ *     NaN or infinity in one token's k or v can reach the outputs of the adjacent group's tokens.
  *   - Device-side waits are bounded.  If one ever expires the kernel records where, stops cleanly,
  *     and s2a_device_status() reports it; outputs of that launch are then undefined.
  */
@@ -42,7 +48,8 @@ extern "C" {
 typedef enum s2a_status {
     S2A_OK = 0,
     S2A_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, N % G, odd G or H, H % Hkv, misaligned pointer, small workspace */
-    S2A_ERR_UNSUPPORTED = -2, /* d not in {64,128}, G not a multiple of 256, device is not sm_100 */
+    S2A_ERR_UNSUPPORTED = -2, /* d not in {64,128}, G or shift not a multiple of 4 tokens (G/2 for the default shift), N < 128,
+                                 ragged tiles with mixed shifts on one KV head, device is not sm_100 */
     S2A_ERR_CUDA = -3,        /* a CUDA call failed while enqueuing; see s2a_last_cuda_error() */
     S2A_ERR_TIMEOUT = -4,     /* reported by s2a_device_status(): a bounded device-side wait expired */
     S2A_ERR_TOO_LARGE = -5    /* s2a_bwd_noalloc only: B*H*N is more than its built-in scratch holds */
@@ -78,8 +85,9 @@ size_t s2a_bwd_workspace_bytes(int B, int N, int H, int Hkv, int d, int G);
 /*
  * Generalised forms (Section 3.2 pilot study, Table 6 and Appendix B variants 1 and 2): the first
  * `n_unshifted` heads use the unshifted partition, the remaining heads are rolled by -shift
- * tokens (shift a multiple of 128, |shift| < N; the paper's method is n_unshifted = H/2,
- * shift = G/2).  n_unshifted = H gives "pattern 1 only"; with G = N as well it is ordinary full
+ * tokens (G and shift multiples of 4, |shift| < N; the paper's method is n_unshifted = H/2,
+ * shift = G/2).  When G or shift is not a multiple of 128 the query heads of one KV head must all be
+ * on the same side of n_unshifted (n_unshifted a multiple of H/Hkv).  n_unshifted = H gives "pattern 1 only"; with G = N as well it is ordinary full
  * causal attention, which the fine-tuned model uses at inference.  `scale` multiplies the scores
  * (pass 1/sqrt(d) for the standard choice).  H may be odd here.
  * flags: S2A_FLAG_LEAK_FREE selects variant 2 of Appendix B ("individual groups for the shifted

@@ -224,12 +224,14 @@ def s2a_fwd_ex(q, k, v, G, scale=None, n_unshifted=None, shift=None, leak_free=F
 
 
 def s2a_bwd_ex(q, k, v, o, lse, dO, G, scale=None, n_unshifted=None, shift=None, leak_free=False, workspace=None,
-               stream=None):
+               stream=None, dq=None, dk=None, dv=None):
     B, N, H, Hkv, d = _dims(q, k)
     scale = 1.0 / math.sqrt(d) if scale is None else scale
     n_unshifted = H // 2 if n_unshifted is None else n_unshifted
     shift = G // 2 if shift is None else shift
-    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(v) if dv is None else dv
     need = bwd_workspace_bytes(B, N, H, Hkv, d, G)
     if workspace is None:
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)

@@ -96,10 +96,22 @@ int check_shape(int B, int N, int H, int Hkv, int d, int G, float scale, int n_u
     if (!(scale > 0.f) || !isfinite(scale)) return S2A_ERR_INVALID_ARG;
     if (shift <= -N || shift >= N) return S2A_ERR_INVALID_ARG;
     if (d != 64 && d != 128) return S2A_ERR_UNSUPPORTED;
-    if (G % kTile != 0 || shift % kTile != 0) return S2A_ERR_UNSUPPORTED;
+    // Every run of tokens of a group must start and end on a multiple of 4 tokens (16 bytes of the
+    // fp32 row statistics, which travel by bulk copies); a tensor map wants at least one whole box.
+    if (G % 4 != 0 || shift % 4 != 0 || N < kTile) return S2A_ERR_UNSUPPORTED;
+    // Ragged tiles (G or shift not a multiple of 128): the key tiles of a KV head follow the partition
+    // of its query heads, which must then all have the same shift.
+    if ((G % kTile != 0 || shift % kTile != 0) && n_unshifted % (H / Hkv) != 0) return S2A_ERR_UNSUPPORTED;
     // grid sizes and 32-bit token arithmetic
-    const long long tiles = (long long)B * H * (N / kTile);
+    const long long tiles = (long long)B * H * (N / G) * (G / kTile + 2);
     if (tiles > 0x7fffffffLL || (long long)N + G >= 0x40000000LL) return S2A_ERR_UNSUPPORTED;
+    return S2A_OK;
+}
+
+// Shape rules of the default entry points (shift G/2 on the second half of the heads).
+int check_default_shape(int N, int H, int d, int G) {
+    if (d <= 0 || H <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
+    if (G % 8 != 0) return (G > 0 && N > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
     return S2A_OK;
 }
 
@@ -108,9 +120,18 @@ Geometry make_geometry(int B, int N, int H, int Hkv, int G, int n_unshifted, int
     g.B = B, g.N = N, g.H = H, g.Hkv = Hkv, g.G = G;
     g.n_unshifted = n_unshifted;
     g.shift = shift;
-    g.tiles_per_group = G / kTile;
     g.groups = N / G;
     g.leak_free = leak_free;
+    // the grid has one slot per (unit, tile rank); groups with fewer tiles leave their last slots idle
+    g.tiles_per_group = 0;
+    const int shifts[2] = {0, shift};
+    for (int which = 0; which < 2; ++which) {
+        if ((which == 0 && n_unshifted == 0) || (which == 1 && n_unshifted == H)) continue;
+        for (int grp = 0; grp < g.groups; ++grp) {
+            const int n = group_layout(g, shifts[which], grp).nTiles;
+            if (n > g.tiles_per_group) g.tiles_per_group = n;
+        }
+    }
     return g;
 }
 
@@ -132,7 +153,7 @@ const char* s2a_status_string(int status) {
     switch (status) {
         case S2A_OK: return "ok";
         case S2A_ERR_INVALID_ARG: return "invalid argument (null or misaligned pointer, bad size, or workspace too small)";
-        case S2A_ERR_UNSUPPORTED: return "unsupported shape or device (need d in {64,128}, G and shift multiples of 128, sm_100)";
+        case S2A_ERR_UNSUPPORTED: return "unsupported shape or device (need d in {64,128}, G and shift multiples of 4 tokens, N >= 128, sm_100)";
         case S2A_ERR_CUDA: return "a CUDA call failed; see s2a_last_cuda_error()";
         case S2A_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case S2A_ERR_TOO_LARGE: return "B*H*N exceeds the built-in scratch of s2a_bwd_noalloc (see s2a_bwd_noalloc_max_rows)";
@@ -179,8 +200,7 @@ int s2a_fwd_ex(const void* q, const void* k, const void* v, void* o, float* lse,
 
 int s2a_fwd_packed(const void* qkv, void* o, float* lse, int B, int N, int H, int d, int G, void* stream) {
     if (!qkv) return S2A_ERR_INVALID_ARG;
-    if (d <= 0 || H <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
-    if (G % (2 * kTile) != 0) return (G > 0 && N > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
+    if (const int bad = check_default_shape(N, H, d, G)) return bad;
     const __nv_bfloat16* base = static_cast<const __nv_bfloat16*>(qkv);
     const long long hd = static_cast<long long>(H) * d;
     TokStrides ts;
@@ -191,8 +211,7 @@ int s2a_fwd_packed(const void* qkv, void* o, float* lse, int B, int N, int H, in
 
 int s2a_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int N, int H, int Hkv, int d,
             int G, void* stream) {
-    if (d <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
-    if (G % (2 * kTile) != 0) return (G > 0 && N > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
+    if (const int bad = check_default_shape(N, H, d, G)) return bad;
     return s2a_fwd_ex(q, k, v, o, lse, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2, G / 2, 0u, stream);
 }
 
@@ -278,8 +297,7 @@ int s2a_bwd_ex(const void* q, const void* k, const void* v, const void* o, const
 int s2a_bwd_packed(const void* qkv, const void* o, const float* lse, const void* dO, void* dqkv, int B, int N, int H,
                    int d, int G, void* workspace, size_t workspace_bytes, void* stream) {
     if (!qkv || !dqkv) return S2A_ERR_INVALID_ARG;
-    if (d <= 0 || H <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
-    if (G % (2 * kTile) != 0) return (G > 0 && N > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
+    if (const int bad = check_default_shape(N, H, d, G)) return bad;
     const __nv_bfloat16* in = static_cast<const __nv_bfloat16*>(qkv);
     __nv_bfloat16* out = static_cast<__nv_bfloat16*>(dqkv);
     const long long hd = static_cast<long long>(H) * d;
@@ -293,8 +311,7 @@ int s2a_bwd_stage(const void* q, const void* k, const void* v, const void* o, co
                   void* dq, void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, void* workspace,
                   size_t workspace_bytes, int stage, void* stream) {
     if (stage < 0 || stage > 2) return S2A_ERR_INVALID_ARG;
-    if (d <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
-    if (G % (2 * kTile) != 0) return (G > 0 && N > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
+    if (const int bad = check_default_shape(N, H, d, G)) return bad;
     return bwd_impl(q, k, v, o, lse, dO, dq, dk, dv, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2,
                     G / 2, workspace, workspace_bytes, stream, 1u << stage);
 }
@@ -302,8 +319,7 @@ int s2a_bwd_stage(const void* q, const void* k, const void* v, const void* o, co
 int s2a_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO, void* dq,
             void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, void* workspace, size_t workspace_bytes,
             void* stream) {
-    if (d <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
-    if (G % (2 * kTile) != 0) return (G > 0 && N > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
+    if (const int bad = check_default_shape(N, H, d, G)) return bad;
     return s2a_bwd_ex(q, k, v, o, lse, dO, dq, dk, dv, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2,
                       G / 2, 0u, workspace, workspace_bytes, stream);
 }
@@ -314,10 +330,9 @@ int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const vo
                      void* workspace, size_t workspace_bytes, void* stream) {
     if (!h_q || !h_k || !h_v || !h_dO || !h_o || !h_lse || !h_dq || !h_dk || !h_dv) return S2A_ERR_INVALID_ARG;
     if (!d_q || !d_k || !d_v || !d_dO || !d_o || !d_lse || !d_dq || !d_dk || !d_dv) return S2A_ERR_INVALID_ARG;
-    if (d <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
+    if (const int bad = check_default_shape(N, H, d, G)) return bad;
     int rc = check_shape(B, N, H, Hkv, d, G, 1.0f, H / 2, G / 2);
     if (rc != S2A_OK) return rc;
-    if (G % (2 * kTile) != 0) return S2A_ERR_UNSUPPORTED;
     if (!workspace || workspace_bytes < s2a_bwd_workspace_bytes(B, N, H, Hkv, d, G)) return S2A_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t nq = static_cast<size_t>(B) * N * H * d * 2;
@@ -378,8 +393,7 @@ int s2a_bwd_noalloc(const void* q, const void* k, const void* v, const void* o, 
     if (static_cast<unsigned long long>(B) * static_cast<unsigned long long>(H) * static_cast<unsigned long long>(N) >
         kBuiltinScratchRows)
         return S2A_ERR_TOO_LARGE;
-    if (d <= 0 || (H & 1) || (G & 1)) return S2A_ERR_INVALID_ARG;
-    if (G % (2 * kTile) != 0) return (G > 0 && N % G == 0) ? S2A_ERR_UNSUPPORTED : S2A_ERR_INVALID_ARG;
+    if (const int bad = check_default_shape(N, H, d, G)) return bad;
     float* scratch = nullptr;
     const int rc = builtin_scratch(&scratch);
     if (rc != S2A_OK) return rc;

@@ -99,7 +99,7 @@ __device__ __forceinline__ void pack32(const float (&x)[32], uint32_t (&out)[16]
 // Store COLS consecutive fp32 accumulator columns of this thread's tensor-memory lane (times `mul`)
 // as bf16 to `dst`.
 template <int COLS>
-__device__ __forceinline__ void store_acc_cols(uint32_t t_addr, float mul, __nv_bfloat16* dst_row) {
+__device__ __forceinline__ void store_acc_cols(uint32_t t_addr, float mul, __nv_bfloat16* dst_row, bool row_valid) {
 #pragma unroll
     for (int c = 0; c < COLS / 32; ++c) {
         uint32_t r[32];
@@ -113,7 +113,7 @@ __device__ __forceinline__ void store_acc_cols(uint32_t t_addr, float mul, __nv_
             pk.y = pack_bf16(__uint_as_float(r[8 * e + 2]) * mul, __uint_as_float(r[8 * e + 3]) * mul);
             pk.z = pack_bf16(__uint_as_float(r[8 * e + 4]) * mul, __uint_as_float(r[8 * e + 5]) * mul);
             pk.w = pack_bf16(__uint_as_float(r[8 * e + 6]) * mul, __uint_as_float(r[8 * e + 7]) * mul);
-            dst[e] = pk;
+            if (row_valid) dst[e] = pk;
         }
     }
 }
@@ -172,15 +172,18 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
     const int Tg = geo.tiles_per_group;
     int unit, rank;
     decode_block(blockIdx.x, geo.B * geo.H * geo.groups, Tg, &unit, &rank);
-    const int i = Tg - 1 - rank;  // heaviest query tiles first
     const int g = unit % geo.groups;
     const int h = (unit / geo.groups) % geo.H;
     const int b = unit / (geo.groups * geo.H);
     const int hk = h / (geo.H / geo.Hkv);
     const int s = (h < geo.n_unshifted) ? 0 : geo.shift;
-    const int n_begin = 2 * first_key_tile(geo, s, g, i);
+    const GroupLayout L = group_layout(geo, s, g);
+    const int i = L.nTiles - 1 - rank;  // heaviest query tiles first
+    if (i < 0) return;                  // this group has fewer tiles than the largest one
+    const int n_begin = 2 * first_key_tile(L, i);
     const int n_steps = 2 * (i + 1) - n_begin;  // key sub-tiles n_begin .. 2i+1 of the group (n_begin = 0 by default)
-    const int tq0 = mod_pos(g * geo.G + i * kTile + s, geo.N);
+    const TileRef tq = tile_ref(L, i);
+    const int tq0 = tq.tok0;
 
     if (threadIdx.x == 0) {
         mbar_init(&bars->res_full, 1);
@@ -225,7 +228,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
             for (; n < n_steps; ++n) {
                 const int st = n % C::kStages;
                 const uint32_t ph = (n / C::kStages) & 1;
-                const int tk0 = mod_pos(g * geo.G + (n_begin + n) * kSubTile + s, geo.N);
+                const int tk0 = subtile_ref(L, n_begin + n).tok0;
                 if (!mbar_wait(&bars->st_empty[st], ph ^ 1, ctx, kWaitBwdDq + 1)) break;
                 mbar_expect_tx(&bars->st_full[st], C::kStageBytes);
                 uint8_t* sK = sStage + st * C::kStageBytes;
@@ -317,9 +320,12 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         const int half = (warp - 4) >> 2;
         const int row = quad * 32 + lane;
         const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+        // rows past the end of a ragged tile are not part of the group: they are computed on whatever
+        // the box holds there and never stored
+        const bool row_valid = row < tq.valid;
         const size_t stat_idx = (static_cast<size_t>(b) * geo.H + h) * geo.N + tq0 + row;
-        const float neg_lse2 = -p.lse[stat_idx] * kLog2e;
-        const float Drow = p.Dsum[stat_idx];
+        const float neg_lse2 = row_valid ? -p.lse[stat_idx] * kLog2e : 0.f;
+        const float Drow = row_valid ? p.Dsum[stat_idx] : 0.f;
         const float c2 = p.scale_log2;
         bool ok = true;
         for (int n = 0; n < n_steps; ++n) {
@@ -333,10 +339,15 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
             tmem_ld_32x32(tP, pr);
             tmem_wait_ld();
             uint32_t pk[16];
-            if (n_begin + n >= 2 * i) {
-                // diagonal sub-tiles: key x of sub-tile m is visible to query row r iff 64 m + x <= 128 i + r
+            const int m = n_begin + n;
+            const int k_valid = subtile_ref(L, m).valid;
+            if (m >= 2 * i || k_valid < kSubTile) {
+                // masked sub-tiles: key x of sub-tile m is visible to query row r iff it is a valid row
+                // and, in the diagonal tile, 64 m + x <= 128 i + r
                 float ds[32];
-                const int lim = i * kTile + row - (n_begin + n) * kSubTile - half * 32;  // visible iff e <= lim
+                int vis = k_valid - 1;
+                if (m >= 2 * i && row - (m & 1) * kSubTile < vis) vis = row - (m & 1) * kSubTile;
+                const int lim = vis - half * 32;  // visible iff e <= lim
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
                     float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, neg_lse2));
@@ -367,7 +378,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDq + 6)) {
             tc_fence_after();
             __nv_bfloat16* dst = p.dq + (static_cast<size_t>(b) * geo.N + tq0 + row) * p.dq_tok_stride + static_cast<size_t>(h) * HD;
-            store_acc_cols<HD / 2>(t_row + kColAcc + half * (HD / 2), p.scale, dst + half * (HD / 2));
+            store_acc_cols<HD / 2>(t_row + kColAcc + half * (HD / 2), p.scale, dst + half * (HD / 2), row_valid);
         }
     }
 
@@ -387,18 +398,22 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
 //
 // The CTA owns key tile (b, hk, original tokens tk0 .. tk0+127).  For every query head hq that
 // reads KV head hk (shift s): the tile sits at rolled position (tk0 - s) mod N, i.e. in group g at
-// key tile j, and is attended by query sub-tiles (64 rows) 2j .. 2*Tg-1 of that group.
+// key tile j, and is attended by query sub-tiles (64 rows) 2j .. 2*nTiles-1 of that group.  (When the
+// tiles are ragged the host only admits KV heads whose query heads all have the same shift, so the
+// key tile is a tile of every head's partition.)
 struct HeadWalk {
-    int s, g, j, n_begin, n_end;
+    GroupLayout L;
+    int j, n_begin, n_end;
 };
 __device__ __forceinline__ HeadWalk head_walk(const Geometry& geo, int hq, int tk0) {
     HeadWalk w;
-    w.s = (hq < geo.n_unshifted) ? 0 : geo.shift;
-    const int pos = mod_pos(tk0 - w.s, geo.N);
-    w.g = pos / geo.G;
-    w.j = (pos % geo.G) / kTile;
+    const int s = (hq < geo.n_unshifted) ? 0 : geo.shift;
+    const int pos = mod_pos(tk0 - s, geo.N);
+    w.L = group_layout(geo, s, pos / geo.G);
+    const int in_group = pos % geo.G;
+    w.j = in_group < w.L.lenA ? in_group / kTile : w.L.nA + (in_group - w.L.lenA) / kTile;
     w.n_begin = 2 * w.j;
-    w.n_end = 2 * end_query_tile(geo, w.s, w.g, w.j);
+    w.n_end = 2 * end_query_tile(w.L, w.j);
     return w;
 }
 
@@ -436,7 +451,10 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
     const int b = unit / (geo.groups * geo.Hkv);
     const int hq0 = hk * rep;
     const int s0 = (hq0 < geo.n_unshifted) ? 0 : geo.shift;
-    const int tk0 = mod_pos(g0 * geo.G + j0 * kTile + s0, geo.N);
+    const GroupLayout L0 = group_layout(geo, s0, g0);
+    if (j0 >= L0.nTiles) return;  // this group has fewer tiles than the largest one
+    const TileRef tk = tile_ref(L0, j0);
+    const int tk0 = tk.tok0;
 
     int total_steps = 0;
     for (int hq = hq0; hq < hq0 + rep; ++hq) {
@@ -490,9 +508,13 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                 for (int n = w.n_begin; n < w.n_end; ++n, ++it) {
                     const int st = it % C::kStages;
                     const uint32_t ph = (it / C::kStages) & 1;
-                    const int tq0 = mod_pos(w.g * geo.G + n * kSubTile + w.s, geo.N);
+                    const TileRef tq = subtile_ref(w.L, n);
+                    const int tq0 = tq.tok0;
+                    // statistics of the valid rows only (a multiple of 4 rows, so of 16 bytes): a ragged
+                    // sub-tile must not read past the end of the arrays
+                    const uint32_t stat_bytes = static_cast<uint32_t>(tq.valid) * 4u;
                     if (!mbar_wait(&bars->st_empty[st], ph ^ 1, ctx, kWaitBwdDkDv + 1)) { ok = false; break; }
-                    mbar_expect_tx(&bars->st_full[st], C::kStageBytes + 2 * C::kStatBytes);
+                    mbar_expect_tx(&bars->st_full[st], C::kStageBytes + 2 * stat_bytes);
                     uint8_t* sQ = sStage + st * C::kStageBytes;
                     uint8_t* sDO = sQ + C::kSubTileBytes;
                     for (int bx = 0; bx < C::kBoxes; ++bx) {
@@ -500,9 +522,10 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                         tma_load_4d(sDO + bx * C::kSubBoxBytes, &p.tm_do, &bars->st_full[st], bx * 64, hq, tq0, b);
                     }
                     const size_t stat_idx = (static_cast<size_t>(b) * geo.H + hq) * geo.N + tq0;
-                    bulk_load_1d(sStat + st * 2 * kSubTile, p.lse + stat_idx, C::kStatBytes, &bars->st_full[st]);
-                    bulk_load_1d(sStat + st * 2 * kSubTile + kSubTile, p.Dsum + stat_idx, C::kStatBytes,
-                                 &bars->st_full[st]);
+                    if (stat_bytes != 0) {
+                        bulk_load_1d(sStat + st * 2 * kSubTile, p.lse + stat_idx, stat_bytes, &bars->st_full[st]);
+                        bulk_load_1d(sStat + st * 2 * kSubTile + kSubTile, p.Dsum + stat_idx, stat_bytes, &bars->st_full[st]);
+                    }
                 }
             }
             if (bars->abort_flag != 0) {
@@ -614,10 +637,14 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                 tmem_ld_32x32(tP, pr);
                 tmem_wait_ld();
                 uint32_t pkP[16], pkS[16];
-                // query x of this sub-tile sees key row r iff 128 j + r <= 64 n + x
-                if (n < w.n_begin + 2) {
-                    // diagonal sub-tiles: scalar path with the mask
-                    const int lim = w.j * kTile + row - n * kSubTile - half * 32;  // visible iff e >= lim
+                // query x of this sub-tile sees key row r iff x is a valid row of the sub-tile and, in the
+                // diagonal tile, 128 j + r <= 64 n + x
+                const int q_valid = subtile_ref(w.L, n).valid;
+                if (n < w.n_begin + 2 || q_valid < kSubTile) {
+                    // masked sub-tiles: scalar path.  Statistics of rows that are not valid were never
+                    // loaded, so a masked entry is set to zero, never multiplied by zero.
+                    const int lim = (n < w.n_begin + 2) ? row - (n & 1) * kSubTile - half * 32 : -64;  // visible iff lim <= e < hi
+                    const int hi = q_valid - half * 32;
                     float pt[32], ds[32];
 #pragma unroll
                     for (int e4 = 0; e4 < 8; ++e4) {
@@ -628,10 +655,10 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
                             const int e = e4 * 4 + u;
-                            float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, -lv[u] * kLog2e));
-                            if (e < lim) pe = 0.f;
-                            pt[e] = pe;
-                            ds[e] = pe * (__uint_as_float(pr[e]) - dv[u]);
+                            const bool visible = (e >= lim) && (e < hi);
+                            const float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, -lv[u] * kLog2e));
+                            pt[e] = visible ? pe : 0.f;
+                            ds[e] = visible ? pe * (__uint_as_float(pr[e]) - dv[u]) : 0.f;
                         }
                     }
                     pack32(pt, pkP);
@@ -671,8 +698,9 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDkDv + 7)) {
             tc_fence_after();
             const size_t out_row = (static_cast<size_t>(b) * geo.N + tk0 + row) * p.dkv_tok_stride + static_cast<size_t>(hk) * HD;
-            if (half == 0) store_acc_cols<HD>(t_row + kColDV, 1.0f, p.dv + out_row);
-            else store_acc_cols<HD>(t_row + kColDK, p.scale, p.dk + out_row);
+            const bool row_valid = row < tk.valid;  // rows past the end of a ragged tile belong to other tiles
+            if (half == 0) store_acc_cols<HD>(t_row + kColDV, 1.0f, p.dv + out_row, row_valid);
+            else store_acc_cols<HD>(t_row + kColDK, p.scale, p.dk + out_row, row_valid);
         }
     }
 

@@ -2,11 +2,14 @@
 //
 // One CTA computes one 128-row query tile of one (batch, head, group): steps "roll", "group",
 // "attention" and "roll back" of Algorithm 1 collapse into the choice of TMA coordinates.  Query
-// tile i of rolled group g in a head with shift s covers ORIGINAL tokens
-// ((g*G + i*128 + s) mod N) .. +127 (s and G are multiples of 128, so a tile never straddles the
-// sequence end); its keys are tiles 0..i of the same group, fetched at their own original
-// positions -- for the wrapped last group of a shifted head that is the range [N-G/2, N) followed
-// by [0, G/2).  Outputs are stored at the original token rows, which is the roll back.
+// tile i of rolled group g in a head with shift s covers the ORIGINAL tokens given by tile_ref():
+// a group is one run of original tokens starting at (g*G + s) mod N, or, where it wraps past the
+// sequence end, two runs ([N-G/2, N) followed by [0, G/2) in Algorithm 1), and each run is tiled from
+// its own start, so a tile never straddles the sequence end.  Its keys are tiles 0..i of the same
+// group, fetched at their own original positions.  When G or s is not a multiple of 128 the last
+// tile of a run has fewer than 128 valid rows: the rest of the box holds neighbouring tokens (or
+// zero fill), masked as key columns and not stored as query rows.  Outputs are stored at the
+// original token rows, which is the roll back.
 //
 // Warp roles (320 threads): warp 0 issues TMA loads, warp 1 owns tensor memory and issues the
 // tcgen05 MMAs, warps 2-9 run the online softmax: a score row lives in one tensor-memory lane
@@ -76,20 +79,18 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
     const int Tg = p.geo.tiles_per_group;
     int unit, it;
     decode_block(blockIdx.x, p.geo.B * p.geo.H * p.geo.groups, Tg, &unit, &it);
-    const int i = Tg - 1 - it;                 // query tile inside the group
     const int g = unit % p.geo.groups;
     const int h = (unit / p.geo.groups) % p.geo.H;
     const int b = unit / (p.geo.groups * p.geo.H);
     const int hk = h / (p.geo.H / p.geo.Hkv);
     const int s = (h < p.geo.n_unshifted) ? 0 : p.geo.shift;
-    const int j_begin = first_key_tile(p.geo, s, g, i);
+    const GroupLayout L = group_layout(p.geo, s, g);
+    const int i = L.nTiles - 1 - it;           // query tile inside the group
+    if (i < 0) return;                         // this group has fewer tiles than the largest one
+    const int j_begin = first_key_tile(L, i);
     const int n_kv = i + 1 - j_begin;          // causal: key tiles j_begin..i of the same group (j_begin = 0 by default)
-    // original token of rolled position x:  (x + s) mod N
-    auto orig_token = [&](int rolled) {
-        int t = (rolled + s) % p.geo.N;
-        return t < 0 ? t + p.geo.N : t;
-    };
-    const int tq0 = orig_token(g * p.geo.G + i * kTile);
+    const TileRef tq = tile_ref(L, i);
+    const int tq0 = tq.tok0;
 
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
@@ -132,7 +133,7 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
             for (; j < n_kv; ++j) {
                 const int st = j % C::kStages;
                 const uint32_t ph = (j / C::kStages) & 1;
-                const int tk0 = orig_token(g * p.geo.G + (j_begin + j) * kTile);
+                const int tk0 = tile_ref(L, j_begin + j).tok0;
                 if (!mbar_wait(k_empty + st, ph ^ 1, ctx, kWaitFwd + 1)) break;
                 mbar_expect_tx(k_full + st, C::kTileBytes);
                 for (int bx = 0; bx < C::kBoxes; ++bx)
@@ -250,8 +251,13 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
             tc_fence_after();
             // pass 1: row maximum of this thread's 64 columns (the scores are read again in pass 2,
             // 32 at a time, which keeps the register footprint small enough for two CTAs per SM)
-            const bool diagonal = (j == n_kv - 1);    // key x of the tile is visible to query row r iff x <= r
-            const int lim = row - half * 64;   // visible iff (column within this half) <= lim
+            // Key x of the tile is visible to query row r iff it is one of the tile's valid rows and,
+            // on the diagonal tile, x <= r.  Off the diagonal a full tile needs no mask at all.
+            const int k_valid = tile_ref(L, j_begin + j).valid;
+            const bool last = (j == n_kv - 1);
+            const bool diagonal = last || k_valid < kTile;   // "this tile is masked"
+            const int vis = (last && row < k_valid) ? row : k_valid - 1;
+            const int lim = vis - half * 64;   // visible iff (column within this half) <= lim
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
@@ -329,6 +335,7 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
             const float l_row = l + l_other;
             const float inv_l = 1.0f / l_row;
             const int t = tq0 + row;
+            const bool row_valid = row < tq.valid;   // rows past the end of a ragged tile are not part of the group
             __nv_bfloat16* orow = p.o + ((static_cast<size_t>(b) * p.geo.N + t) * p.geo.H + h) * HD + half * (HD / 2);
 #pragma unroll
             for (int c = 0; c < HD / 64; ++c) {
@@ -343,11 +350,11 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
                     pk.y = pack_bf16(__uint_as_float(oreg[8 * e + 2]) * inv_l, __uint_as_float(oreg[8 * e + 3]) * inv_l);
                     pk.z = pack_bf16(__uint_as_float(oreg[8 * e + 4]) * inv_l, __uint_as_float(oreg[8 * e + 5]) * inv_l);
                     pk.w = pack_bf16(__uint_as_float(oreg[8 * e + 6]) * inv_l, __uint_as_float(oreg[8 * e + 7]) * inv_l);
-                    dst[e] = pk;
+                    if (row_valid) dst[e] = pk;
                 }
             }
             // natural-log sum-exp of the scaled scores
-            if (half == 0)
+            if (half == 0 && row_valid)
                 p.lse[(static_cast<size_t>(b) * p.geo.H + h) * p.geo.N + t] = (m_used + log2f(l_row)) * 0.6931471805599453f;
         }
     }

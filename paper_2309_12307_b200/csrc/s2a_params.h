@@ -39,33 +39,66 @@ struct Geometry {
     int B, N, H, Hkv, G;
     int n_unshifted;      // heads [0, n_unshifted) use the unshifted partition
     int shift;            // tokens; the rest of the heads are rolled by -shift (G/2 in Algorithm 1)
-    int tiles_per_group;  // G / 128
+    int tiles_per_group;  // largest number of 128-token tiles any group has (G / 128 when G and shift are multiples of 128)
     int groups;           // N / G
     int leak_free;        // variant 2 of Appendix B: cut the wrapped group of a shifted head at the wrap
 };
 
-// Variant 2: in a head with shift s != 0 the group that contains the rolled position of original
-// token 0 (pw = -s mod N) is cut in two there; queries at or after the cut attend keys from the cut
-// on, keys before the cut are attended by queries before the cut only.  Both in units of 128-token
-// tiles inside the group; without the variant they are 0 and tiles_per_group.
-__host__ __device__ inline int first_key_tile(const Geometry& geo, int s, int g, int i) {
-    if (geo.leak_free && s != 0) {
-        int pw = (-s) % geo.N;
-        if (pw < 0) pw += geo.N;
-        const int iw = (pw % geo.G) / kTile;
-        if (g == pw / geo.G && iw > 0 && i >= iw) return iw;
-    }
-    return 0;
+// Where the tokens of one group live.  Group g of a head with shift s holds rolled positions
+// [g G, (g+1) G), i.e. original tokens (x + s) mod N: one run [a0, a0 + lenA) and, only in the group
+// that wraps past token N-1, a second run [0, lenB).  Each run is cut into 128-token tiles from its own
+// start, so a tile is always a contiguous range of original tokens (one TMA box, no wrap inside a
+// tile) and only the last tile of a run can have fewer than 128 valid rows.  Tiles are numbered in
+// rolled (= causal) order: the nA tiles of the first run, then those of the second.
+struct GroupLayout {
+    int a0, lenA, lenB;
+    int nA, nTiles;
+    int cut;  // variant 2: tile index at which the wrapped group is cut in two (0 = no cut)
+};
+__host__ __device__ inline GroupLayout group_layout(const Geometry& geo, int s, int g) {
+    GroupLayout L;
+    long long a = (static_cast<long long>(g) * geo.G + s) % geo.N;
+    if (a < 0) a += geo.N;
+    L.a0 = static_cast<int>(a);
+    L.lenA = (geo.N - L.a0 < geo.G) ? geo.N - L.a0 : geo.G;
+    L.lenB = geo.G - L.lenA;
+    L.nA = (L.lenA + kTile - 1) / kTile;
+    L.nTiles = L.nA + (L.lenB + kTile - 1) / kTile;
+    // Variant 2: the second run starts at original token 0; queries there attend keys from the cut
+    // on, keys before the cut are attended by queries before the cut only.
+    L.cut = (geo.leak_free && L.lenB > 0) ? L.nA : 0;
+    return L;
 }
-__host__ __device__ inline int end_query_tile(const Geometry& geo, int s, int g, int j) {
-    if (geo.leak_free && s != 0) {
-        int pw = (-s) % geo.N;
-        if (pw < 0) pw += geo.N;
-        const int iw = (pw % geo.G) / kTile;
-        if (g == pw / geo.G && iw > 0 && j < iw) return iw;
+struct TileRef {
+    int tok0;   // original token of row 0
+    int valid;  // rows that belong to the group (the rest of the box is other tokens or zero fill)
+};
+__host__ __device__ inline TileRef tile_ref(const GroupLayout& L, int i) {
+    TileRef t;
+    if (i < L.nA) {
+        t.tok0 = L.a0 + i * kTile;
+        t.valid = L.lenA - i * kTile;
+    } else {
+        t.tok0 = (i - L.nA) * kTile;
+        t.valid = L.lenB - (i - L.nA) * kTile;
     }
-    return geo.tiles_per_group;
+    if (t.valid > kTile) t.valid = kTile;
+    return t;
 }
+// 64-row halves of the tiles, numbered 2 i and 2 i + 1; a half can be empty (valid = 0).
+__host__ __device__ inline TileRef subtile_ref(const GroupLayout& L, int n) {
+    TileRef t = tile_ref(L, n >> 1);
+    const int off = (n & 1) * kSubTile;
+    t.tok0 += off;
+    t.valid -= off;
+    if (t.valid > kSubTile) t.valid = kSubTile;
+    if (t.valid < 0) t.valid = 0;
+    return t;
+}
+// Causal range in tiles: query tile i attends key tiles [first_key_tile, i]; key tile j is attended
+// by query tiles [j, end_query_tile).
+__host__ __device__ inline int first_key_tile(const GroupLayout& L, int i) { return (L.cut > 0 && i >= L.cut) ? L.cut : 0; }
+__host__ __device__ inline int end_query_tile(const GroupLayout& L, int j) { return (L.cut > 0 && j < L.cut) ? L.cut : L.nTiles; }
 
 struct alignas(64) FwdParams {
     CUtensorMap tm_q;  // bf16 (d, H,   N, B), box (64, 1, 128, 1), 128-byte swizzle

@@ -52,6 +52,12 @@ WORKLOADS = {
     "llama2_7b_32k": Workload("llama2_7b_32k", 1, 32768, 8192, 32, 32, 128),
     "llama2_7b_100k": Workload("llama2_7b_100k", 1, 102400, 25600, 32, 32, 128),
     "llama2_70b_32k_gqa": Workload("llama2_70b_32k_gqa", 1, 32768, 8192, 64, 8, 128),
+    # further context lengths and model sizes of Tables 3-4 (G = N/4 throughout)
+    "llama2_7b_16k": Workload("llama2_7b_16k", 1, 16384, 4096, 32, 32, 128),
+    "llama2_7b_64k": Workload("llama2_7b_64k", 1, 65536, 16384, 32, 32, 128),
+    "llama2_13b_32k": Workload("llama2_13b_32k", 1, 32768, 8192, 40, 40, 128),
+    # the literal 100,000-token context: G = 25,000 and G/2 = 12,500 are not multiples of the 128-token tile
+    "llama2_7b_100000": Workload("llama2_7b_100000", 1, 100000, 25000, 32, 32, 128),
 }
 
 

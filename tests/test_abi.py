@@ -80,10 +80,11 @@ def test_bad_arguments_are_rejected_without_a_device(lib):
     assert lib.s2a_fwd(a, a, a, a, a, 1, 1024, 3, 3, 64, 256, None) == -1
     assert lib.s2a_fwd(a, a, a, a, a, 1, 1023, 4, 4, 64, 341, None) == -1
     assert lib.s2a_fwd(a, a, a, a, a, 1, 1024, 4, 3, 64, 256, None) == -1
-    # unsupported: head dim, group size not a multiple of 256
+    # unsupported: head dim, half a group not a multiple of 4 tokens, sequence shorter than one tile
     assert lib.s2a_fwd(a, a, a, a, a, 1, 1024, 4, 4, 96, 256, None) == -2
-    assert lib.s2a_fwd(a, a, a, a, a, 1, 1024, 4, 4, 64, 128, None) == -2
-    assert lib.s2a_fwd(a, a, a, a, a, 1, 1200, 4, 4, 64, 200, None) == -2
+    assert lib.s2a_fwd(a, a, a, a, a, 1, 1200, 4, 4, 64, 100, None) == -2
+    assert lib.s2a_fwd(a, a, a, a, a, 1, 1212, 4, 4, 64, 404, None) == -2
+    assert lib.s2a_fwd(a, a, a, a, a, 1, 64, 4, 4, 64, 32, None) == -2
     # backward: workspace too small / missing
     lib.s2a_bwd.argtypes = [P] * 9 + [ctypes.c_int] * 6 + [P, ctypes.c_size_t, P]
     assert lib.s2a_bwd(a, a, a, a, a, a, a, a, a, 1, 1024, 4, 4, 64, 256, a, 16, None) == -1

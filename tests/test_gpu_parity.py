@@ -107,6 +107,55 @@ def test_generalised_shift_and_head_split(s2a):
     assert np.abs(o - o_ref).max() <= O_ATOL
 
 
+RAGGED = [
+    # B, N, G, H, Hkv, d, extra     G or G/2 not a multiple of the 128-token tile: ragged last tiles, and the
+    #                               wrapped group of the shifted heads is cut into two runs of tiles
+    (1, 1200, 200, 4, 4, 64, {}),       # two tiles per run (128 + 72), wrapped group 100 + 100
+    (2, 2000, 1000, 4, 2, 128, {}),     # 8 tiles per group (7 x 128 + 104); wrapped group 500 + 500
+    (1, 1536, 384, 4, 1, 64, dict(n_unshifted=0, shift=192)),   # MQA, every head shifted by half a tile more than one tile
+    (1, 1280, 128, 2, 2, 128, {}),      # G = one tile, shift = half a tile
+    (1, 640, 40, 2, 2, 64, {}),         # groups far smaller than a tile
+    (1, 3000, 1000, 4, 4, 128, dict(leak_free=True)),                           # variant 2 with a ragged cut
+    (1, 1200, 600, 4, 2, 64, dict(n_unshifted=2, shift=-300)),                  # other roll direction
+    (1, 1200, 600, 4, 2, 64, dict(n_unshifted=2, shift=44, scale=0.3)),         # arbitrary shift (multiple of 4)
+    (1, 1200, 600, 4, 2, 64, dict(n_unshifted=2, shift=44, leak_free=True)),
+    (1, 904, 904, 2, 2, 64, dict(n_unshifted=2, shift=0)),                      # full causal attention, ragged length
+]
+
+
+@pytest.mark.parametrize("B,N,G,H,Hkv,d,ex", RAGGED)
+def test_ragged_group_sizes_match_oracle_everywhere(s2a, B, N, G, H, Hkv, d, ex):
+    """Group sizes as the paper uses them (G = N/4 of any N, e.g. 25,000 of 100,000) need not be a
+    multiple of the 128-token tile.  Outputs are pre-filled with NaN: every row must be written, by
+    exactly the tile that owns it."""
+    q, k, v, dO = make_inputs(B, N, H, Hkv, d, seed=11)
+    dev = torch.device("cuda:0")
+    qd, kd, vd, dOd = (x.to(dev) for x in (q, k, v, dO))
+    o = torch.full_like(qd, float("nan"))
+    lse = torch.full((B, H, N), float("nan"), dtype=torch.float32, device=dev)
+    dq, dk, dv = torch.full_like(qd, float("nan")), torch.full_like(kd, float("nan")), torch.full_like(vd, float("nan"))
+    if ex:
+        s2a.s2a_fwd_ex(qd, kd, vd, G, o=o, lse=lse, **ex)
+        s2a.s2a_bwd_ex(qd, kd, vd, o, lse, dOd, G, dq=dq, dk=dk, dv=dv, **ex)
+    else:
+        s2a.s2a_fwd(qd, kd, vd, G, o=o, lse=lse)
+        s2a.s2a_bwd(qd, kd, vd, o, lse, dOd, G, dq=dq, dk=dk, dv=dv)
+    torch.cuda.synchronize()
+    assert s2a.device_status()[0] == 0
+    o, lse, dq, dk, dv = (x.float().cpu().numpy().astype(np.float64) for x in (o, lse, dq, dk, dv))
+    o_ref, lse_ref = orc.fwd(q, k, v, G, **ex)
+    dq_ref, dk_ref, dv_ref = orc.bwd(q, k, v, dO, G, **ex)
+    for x in (o, lse, dq, dk, dv):
+        assert np.isfinite(x).all()
+    assert np.abs(o - o_ref).max() <= O_ATOL
+    assert np.abs(lse - lse_ref).max() <= LSE_ATOL
+    for h in range(H):
+        assert rel_l2(dq[:, :, h], dq_ref[:, :, h]) <= GRAD_REL_L2, h
+    for hk in range(Hkv):
+        assert rel_l2(dk[:, :, hk], dk_ref[:, :, hk]) <= GRAD_REL_L2, hk
+        assert rel_l2(dv[:, :, hk], dv_ref[:, :, hk]) <= GRAD_REL_L2, hk
+
+
 def test_leak_free_variant_matches_oracle(s2a):
     """Appendix B, variant 2 on a head-dim-128 GQA shape with eight tiles per group: the wrapped group
     of the shifted heads is cut at the wrap (tile 4 of 8)."""
@@ -201,7 +250,10 @@ def test_guard_bands_stay_intact(s2a):
 def test_runtime_rejections_on_device(s2a):
     q, k, v, dO = (x.cuda() for x in make_inputs(1, 512, 2, 2, 64, seed=4))
     with pytest.raises(s2a.S2AError) as e:
-        s2a.s2a_fwd(q, k, v, 128)          # G/2 is not a whole tile
+        s2a.s2a_fwd(*(x[:, :504].contiguous() for x in (q, k, v)), 252)   # G/2 is not a multiple of 4 tokens
+    assert e.value.status == s2a.S2A_ERR_UNSUPPORTED
+    with pytest.raises(s2a.S2AError) as e:
+        s2a.s2a_fwd_ex(q, k[:, :, :1].contiguous(), v[:, :, :1].contiguous(), 128, n_unshifted=1, shift=64)   # ragged tiles, mixed shifts on one KV head
     assert e.value.status == s2a.S2A_ERR_UNSUPPORTED
     with pytest.raises(s2a.S2AError) as e:
         s2a.s2a_fwd(q, k, v, 384)          # N % G
@@ -237,7 +289,8 @@ def _sample_rows(w, kv_tail):
     return q_rows, kv_rows
 
 
-FULL = [("llama2_7b_8k", 2048), ("llama2_7b_32k", 1500), ("llama2_70b_32k_gqa", 600), ("llama2_7b_100k", 700)]
+FULL = [("llama2_7b_8k", 2048), ("llama2_7b_32k", 1500), ("llama2_70b_32k_gqa", 600), ("llama2_7b_100k", 700),
+        ("llama2_7b_16k", 1500), ("llama2_7b_64k", 900), ("llama2_13b_32k", 1500), ("llama2_7b_100000", 700)]
 
 
 @pytest.mark.parametrize("name,kv_tail", FULL)

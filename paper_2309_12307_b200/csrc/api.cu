@@ -249,8 +249,8 @@ int bwd_impl(const void* q, const void* k, const void* v, const void* o, const f
     memset(&pq, 0, sizeof pq);
     if ((rc = make_tmap(&pq.tm_q, q, d, H, N, B, kTile, ts.q)) != S2A_OK) return rc;
     if ((rc = make_tmap(&pq.tm_do, dO, d, H, N, B, kTile)) != S2A_OK) return rc;
-    if ((rc = make_tmap(&pq.tm_k, k, d, Hkv, N, B, kSubTile, ts.kv)) != S2A_OK) return rc;
-    if ((rc = make_tmap(&pq.tm_v, v, d, Hkv, N, B, kSubTile, ts.kv)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pq.tm_k, k, d, Hkv, N, B, kTile, ts.kv)) != S2A_OK) return rc;
+    if ((rc = make_tmap(&pq.tm_v, v, d, Hkv, N, B, kTile, ts.kv)) != S2A_OK) return rc;
     pq.dq_tok_stride = ts.dq ? ts.dq : static_cast<long long>(H) * d;
     pq.lse = lse, pq.Dsum = Dsum, pq.dq = static_cast<__nv_bfloat16*>(dq);
     pq.status = ds->status_ptr, pq.geo = geo, pq.scale = scale, pq.scale_log2 = scale * kLog2eHost;

@@ -143,20 +143,57 @@ struct BwdBars {
 // ------------------------------------------------------------------------------------------------
 // 2. dQ
 // ------------------------------------------------------------------------------------------------
-// Tensor memory columns: dQ [0,HD)   three S buffers [128,320)   three dP buffers [320,512)
-// (three score buffers in flight: the chain scores -> elementwise -> dQ MMA of one buffer is about
-// twice as long as the tensor-pipe work of a step, so two buffers leave the pipe idle)
+// One CTA per 128-row query tile; it walks the 128-key tiles j_begin..i of its group (keys <= query).
+// Per key tile n:  S_n = Q K_n^T,  dP_n = dO V_n^T,  dS_n = P_n o (dP_n - D) as bf16 written over the
+// start of S_n's columns,  dQ += dS_n K_n  (K_n is MN-major in the tile that served Q K_n^T).
+// Full 128x128 score products: a 64-column product re-reads the 128-row A operand from shared memory
+// for half the work and runs at 48 instead of 32 clocks per K step.
+//
+// Tensor memory columns: dQ [0,HD)   S buffers [128,256) [256,384)   dP [384,512)
+// Only one dP buffer fits, so the elementwise warps first copy their part of dP_n into registers and
+// release the buffer at once: dP_{n+1} (and S_{n+1}, into the other S buffer) run while they work on
+// step n.  Shared memory: Q_i and dO_i resident, a ring of three K tiles and a ring of two V tiles.
 template <int HD>
-__global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(const __grid_constant__ BwdDqParams p) {
-    using C = BwdCfg<HD>;
-    using Bars = BwdBars<C::kStages>;
-    constexpr int kBufs = 3;
+struct DqCfg {
+    static constexpr int kThreads = 384;  // TMA warp, two MMA warps, one spare, 8 elementwise warps
+    static constexpr int kBoxes = HD / 64;
+    static constexpr int kBoxBytes = kTile * 128;          // 128 rows x 128 bytes
+    static constexpr int kTileBytes = kBoxes * kBoxBytes;  // one Q, dO, K or V tile
+    // K_n serves S_n early in step n-1 and the dQ MMAs at the end of step n: three K tiles are live
+    // around the issue of S_{n+1}, V_n only until dP_n is done.
+    static constexpr int kRingK = 3;
+    static constexpr int kRingV = 2;
+    static constexpr int kBarBytes = 512;
+    static constexpr int kNeeded = 1024 + (2 + kRingK + kRingV) * kTileBytes + kBarBytes;
+    // at least 120 KB so that only one CTA fits on an SM: each CTA allocates all of tensor memory
+    static constexpr int kSmemBytes = kNeeded > 120 * 1024 ? kNeeded : 120 * 1024;
+    static constexpr int kTmemCols = 512;
+};
+
+struct DqBars {
+    uint64_t res_full;     // Q_i and dO_i landed
+    uint64_t acc_full;     // all dQ MMAs done
+    uint64_t drain;        // abort path only (gradient MMA warp)
+    uint64_t drain2;       // abort path only (score MMA warp)
+    uint64_t dp_full;      // S_n and dP_n are in tensor memory
+    uint64_t dp_free;      // every elementwise thread holds its part of dP_n in registers
+    uint64_t p_full[2];    // bf16 dS_n is in tensor memory
+    uint64_t buf_free[2];  // the dQ MMAs that read an S buffer's bf16 dS are done
+    uint64_t k_full[3], k_empty[3], v_full[2], v_empty[2];
+    uint32_t tmem_slot;
+    int abort_flag;
+};
+
+template <int HD>
+__global__ void __launch_bounds__(DqCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(const __grid_constant__ BwdDqParams p) {
+    using C = DqCfg<HD>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem;                                // resident: Q_i
-    uint8_t* sDO = sQ + C::kBigTileBytes;              // resident: dO_i
-    uint8_t* sStage = sDO + C::kBigTileBytes;          // per stage: K_n then V_n
-    Bars* bars = reinterpret_cast<Bars*>(sStage + C::kStages * C::kStageBytes + C::kStages * 2 * C::kStatBytes);
+    uint8_t* sDO = sQ + C::kTileBytes;                 // resident: dO_i
+    uint8_t* sK = sDO + C::kTileBytes;                 // ring of K tiles
+    uint8_t* sV = sK + C::kRingK * C::kTileBytes;      // ring of V tiles
+    DqBars* bars = reinterpret_cast<DqBars*>(sV + C::kRingV * C::kTileBytes);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -180,8 +217,8 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
     const GroupLayout L = group_layout(geo, s, g);
     const int i = L.nTiles - 1 - rank;  // heaviest query tiles first
     if (i < 0) return;                  // this group has fewer tiles than the largest one
-    const int n_begin = 2 * first_key_tile(L, i);
-    const int n_steps = 2 * (i + 1) - n_begin;  // key sub-tiles n_begin .. 2i+1 of the group (n_begin = 0 by default)
+    const int j_begin = first_key_tile(L, i);
+    const int n_steps = i + 1 - j_begin;  // key tiles j_begin .. i of the group (j_begin = 0 by default)
     const TileRef tq = tile_ref(L, i);
     const int tq0 = tq.tok0;
 
@@ -190,14 +227,17 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         mbar_init(&bars->acc_full, 1);
         mbar_init(&bars->drain, 1);
         mbar_init(&bars->drain2, 1);
-        for (int x = 0; x < kBufs; ++x) {
-            mbar_init(&bars->s_full[x], 1);
+        mbar_init(&bars->dp_full, 1);
+        mbar_init(&bars->dp_free, 256);
+        for (int x = 0; x < 2; ++x) {
             mbar_init(&bars->p_full[x], 256);
             mbar_init(&bars->buf_free[x], 1);
+            mbar_init(&bars->v_full[x], 1);
+            mbar_init(&bars->v_empty[x], 1);
         }
-        for (int st = 0; st < C::kStages; ++st) {
-            mbar_init(&bars->st_full[st], 1);
-            mbar_init(&bars->st_empty[st], 1);
+        for (int x = 0; x < C::kRingK; ++x) {
+            mbar_init(&bars->k_full[x], 1);
+            mbar_init(&bars->k_empty[x], 1);
         }
         bars->abort_flag = 0;
         fence_barrier_init();
@@ -215,65 +255,78 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_slot;
     const WaitCtx ctx{&bars->abort_flag, p.status};
-    constexpr uint32_t kColAcc = 0, kColS = 128, kColP = 128 + kBufs * kSubTile;
+    constexpr uint32_t kColAcc = 0, kColS = 128, kColP = 384;
 
     if (warp == 0) {
         if (lane == 0) {
-            mbar_expect_tx(&bars->res_full, 2 * C::kBigTileBytes);
+            mbar_expect_tx(&bars->res_full, 2 * C::kTileBytes);
             for (int bx = 0; bx < C::kBoxes; ++bx) {
-                tma_load_4d(sQ + bx * C::kBigBoxBytes, &p.tm_q, &bars->res_full, bx * 64, h, tq0, b);
-                tma_load_4d(sDO + bx * C::kBigBoxBytes, &p.tm_do, &bars->res_full, bx * 64, h, tq0, b);
+                tma_load_4d(sQ + bx * C::kBoxBytes, &p.tm_q, &bars->res_full, bx * 64, h, tq0, b);
+                tma_load_4d(sDO + bx * C::kBoxBytes, &p.tm_do, &bars->res_full, bx * 64, h, tq0, b);
             }
             int n = 0;
             for (; n < n_steps; ++n) {
-                const int st = n % C::kStages;
-                const uint32_t ph = (n / C::kStages) & 1;
-                const int tk0 = subtile_ref(L, n_begin + n).tok0;
-                if (!mbar_wait(&bars->st_empty[st], ph ^ 1, ctx, kWaitBwdDq + 1)) break;
-                mbar_expect_tx(&bars->st_full[st], C::kStageBytes);
-                uint8_t* sK = sStage + st * C::kStageBytes;
-                uint8_t* sV = sK + C::kSubTileBytes;
-                for (int bx = 0; bx < C::kBoxes; ++bx) {
-                    tma_load_4d(sK + bx * C::kSubBoxBytes, &p.tm_k, &bars->st_full[st], bx * 64, hk, tk0, b);
-                    tma_load_4d(sV + bx * C::kSubBoxBytes, &p.tm_v, &bars->st_full[st], bx * 64, hk, tk0, b);
+                const int st = n & 1;
+                const uint32_t ph = (n >> 1) & 1;
+                const int tk0 = tile_ref(L, j_begin + n).tok0;
+                if (!mbar_wait(&bars->v_empty[st], ph ^ 1, ctx, kWaitBwdDq + 1)) break;
+                mbar_expect_tx(&bars->v_full[st], C::kTileBytes);
+                for (int bx = 0; bx < C::kBoxes; ++bx)
+                    tma_load_4d(sV + st * C::kTileBytes + bx * C::kBoxBytes, &p.tm_v, &bars->v_full[st], bx * 64, hk, tk0, b);
+                const int sk = n % C::kRingK;
+                const uint32_t phk = (n / C::kRingK) & 1;
+                if (!mbar_wait(&bars->k_empty[sk], phk ^ 1, ctx, kWaitBwdDq + 8)) {
+                    mbar_wait_drain(&bars->v_full[st], ph);
+                    break;
                 }
+                mbar_expect_tx(&bars->k_full[sk], C::kTileBytes);
+                for (int bx = 0; bx < C::kBoxes; ++bx)
+                    tma_load_4d(sK + sk * C::kTileBytes + bx * C::kBoxBytes, &p.tm_k, &bars->k_full[sk], bx * 64, hk, tk0, b);
             }
             if (bars->abort_flag != 0) {
+                // let loads that are still in flight land before the CTA gives its memory back
                 mbar_wait_drain(&bars->res_full, 0);
-                for (int nn = (n > C::kStages ? n - C::kStages : 0); nn < n; ++nn)
-                    mbar_wait_drain(&bars->st_full[nn % C::kStages], (nn / C::kStages) & 1);
+                for (int nn = (n > C::kRingK ? n - C::kRingK : 0); nn < n; ++nn)
+                    mbar_wait_drain(&bars->k_full[nn % C::kRingK], (nn / C::kRingK) & 1);
+                for (int nn = (n > C::kRingV ? n - C::kRingV : 0); nn < n; ++nn)
+                    mbar_wait_drain(&bars->v_full[nn & 1], (nn >> 1) & 1);
             }
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ---- score MMAs: S = Q K^T and dP = dO V^T of step n into buffer n % 3.  The whole warp
-        // walks the loop so that addresses and descriptors stay warp-uniform values; only the MMA
-        // and commit instructions themselves are issued by one elected lane.
-        constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);
+        // ---- score MMAs: dP_n = dO V_n^T first (its buffer is free as soon as the elementwise warps
+        // hold dP_{n-1} in registers), then S_n = Q K_n^T into S buffer n & 1 (free once the dQ MMAs
+        // of step n-2 are done).  The whole warp walks the loop so that addresses and descriptors
+        // stay warp-uniform values; only the MMA and commit instructions are issued by one elected lane.
+        constexpr uint32_t idesc_sc = idesc_bf16(128, kTile, 0, 0);
         const uint32_t dQ = desc_lo_k_major(smem_u32(sQ)), dDO = desc_lo_k_major(smem_u32(sDO));
+        const uint32_t tP = tmem_base + kColP;
         bool ok = mbar_wait_uniform(&bars->res_full, 0, ctx, kWaitBwdDq + 3);
         for (int n = 0; ok && n < n_steps; ++n) {
-            const int st = n % C::kStages;
-            if (!mbar_wait_uniform(&bars->st_full[st], (n / C::kStages) & 1, ctx, kWaitBwdDq + 2)) break;
-            const int bf = n % kBufs;
-            const uint32_t use = (n / kBufs) & 1;  // parity of this buffer's use count
-            // the buffer still holds the bf16 dS of step n - 3 until that step's dQ MMAs are done
-            if (n >= kBufs && !mbar_wait_uniform(&bars->buf_free[bf], use ^ 1, ctx, kWaitBwdDq + 7)) break;
+            const int st = n & 1;
+            const uint32_t ph = (n >> 1) & 1;
+            if (!mbar_wait_uniform(&bars->v_full[st], ph, ctx, kWaitBwdDq + 2)) break;
+            if (n >= 1 && !mbar_wait_uniform(&bars->dp_free, (n - 1) & 1, ctx, kWaitBwdDq + 9)) break;
             tc_fence_after();
-            const uint32_t aK = smem_u32(sStage + st * C::kStageBytes);
-            const uint32_t dK = desc_lo_k_major(aK), dV = desc_lo_k_major(aK + C::kSubTileBytes);
-            const uint32_t tS = tmem_base + kColS + bf * kSubTile;
-            const uint32_t tP = tmem_base + kColP + bf * kSubTile;
+            const uint32_t dV = desc_lo_k_major(smem_u32(sV + st * C::kTileBytes));
             if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk)
-                    mma_ss(tS, dQ + desc_step_k_major(kk, C::kBigBoxBytes), dK + desc_step_k_major(kk, C::kSubBoxBytes),
-                           idesc_sc, kk > 0);
+                    mma_ss(tP, dDO + desc_step_k_major(kk, C::kBoxBytes), dV + desc_step_k_major(kk, C::kBoxBytes), idesc_sc, kk > 0);
+                mma_commit(&bars->v_empty[st]);
+            }
+            __syncwarp();
+            const int sk = n % C::kRingK;
+            if (!mbar_wait_uniform(&bars->k_full[sk], (n / C::kRingK) & 1, ctx, kWaitBwdDq + 10)) break;
+            if (n >= 2 && !mbar_wait_uniform(&bars->buf_free[st], ph ^ 1, ctx, kWaitBwdDq + 7)) break;
+            tc_fence_after();
+            const uint32_t dK = desc_lo_k_major(smem_u32(sK + sk * C::kTileBytes));
+            const uint32_t tS = tmem_base + kColS + st * kTile;
+            if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk)
-                    mma_ss(tP, dDO + desc_step_k_major(kk, C::kBigBoxBytes), dV + desc_step_k_major(kk, C::kSubBoxBytes),
-                           idesc_sc, kk > 0);
-                mma_commit(&bars->s_full[bf]);
+                    mma_ss(tS, dQ + desc_step_k_major(kk, C::kBoxBytes), dK + desc_step_k_major(kk, C::kBoxBytes), idesc_sc, kk > 0);
+                mma_commit(&bars->dp_full);  // completes after every MMA issued so far: dP_n and S_n
             }
             __syncwarp();
         }
@@ -285,22 +338,22 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         }
         __syncwarp();
     } else if (warp == 2) {
-        // ---- gradient MMAs: dQ += dS K of step n (K is MN-major in the tile that served Q K^T)
+        // ---- gradient MMAs: dQ += dS_n K_n
         constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);
         for (int n = 0; n < n_steps; ++n) {
-            const int st = n % C::kStages;
-            const int bf = n % kBufs;
-            if (!mbar_wait_uniform(&bars->p_full[bf], (n / kBufs) & 1, ctx, kWaitBwdDq + 4)) break;
+            const int st = n & 1;
+            if (!mbar_wait_uniform(&bars->p_full[st], (n >> 1) & 1, ctx, kWaitBwdDq + 4)) break;
             tc_fence_after();
-            const uint32_t dKmn = desc_lo_mn_major(smem_u32(sStage + st * C::kStageBytes), C::kSubBoxBytes);
-            const uint32_t tdS = tmem_base + kColS + bf * kSubTile;  // bf16 dS over the S buffer
+            const int sk = n % C::kRingK;
+            const uint32_t dKmn = desc_lo_mn_major(smem_u32(sK + sk * C::kTileBytes), C::kBoxBytes);
+            const uint32_t tdS = tmem_base + kColS + st * kTile;  // bf16 dS over the S buffer
             if (elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < kSubTile / 16; ++kk)
-                    mma_ts(tmem_base + kColAcc, tdS + packed_operand_col(kk), dKmn + kk * kDescStepMn, idesc_acc,
+                for (int kk = 0; kk < kTile / 16; ++kk)
+                    mma_ts(tmem_base + kColAcc, tdS + (kk >> 2) * 64 + (kk & 3) * 8, dKmn + kk * kDescStepMn, idesc_acc,
                            (n > 0) || (kk > 0));
-                mma_commit(&bars->st_empty[st]);
-                mma_commit(&bars->buf_free[bf]);
+                mma_commit(&bars->k_empty[sk]);
+                mma_commit(&bars->buf_free[st]);
                 if (n == n_steps - 1) mma_commit(&bars->acc_full);
             }
             __syncwarp();
@@ -316,6 +369,10 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
     } else if (warp == 3) {
         // spare warp: owns the tensor-memory allocation only
     } else {
+        // ---- elementwise: thread (quad, lane, half) owns columns [64 half, +64) of score row
+        // 32 quad + lane.  Its 64 bf16 dS values (32 packed columns) go over the first 32 of its own
+        // columns, so the two halves never write into columns the other half still has to read: the
+        // 128 K values of the dS operand sit at packed columns [0,32) and [64,96) of the S buffer.
         const int quad = warp & 3;
         const int half = (warp - 4) >> 2;
         const int row = quad * 32 + lane;
@@ -327,53 +384,63 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(con
         const float neg_lse2 = row_valid ? -p.lse[stat_idx] * kLog2e : 0.f;
         const float Drow = row_valid ? p.Dsum[stat_idx] : 0.f;
         const float c2 = p.scale_log2;
+        const uint64_t c2x2 = f2_pack(c2, c2), nlx2 = f2_pack(neg_lse2, neg_lse2), Dx2 = f2_pack(Drow, Drow);
         bool ok = true;
         for (int n = 0; n < n_steps; ++n) {
-            const int bf = n % kBufs;
-            if (!mbar_wait(&bars->s_full[bf], (n / kBufs) & 1, ctx, kWaitBwdDq + 5)) { ok = false; break; }
+            const int st = n & 1;
+            if (!mbar_wait(&bars->dp_full, n & 1, ctx, kWaitBwdDq + 5)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t tS = t_row + kColS + bf * kSubTile + half * 32;
-            const uint32_t tP = t_row + kColP + bf * kSubTile + half * 32;
-            uint32_t sr[32], pr[32];
-            tmem_ld_32x32(tS, sr);
-            tmem_ld_32x32(tP, pr);
+            uint32_t dp[64];
+            tmem_ld_32x32(t_row + kColP + half * 64, *reinterpret_cast<uint32_t(*)[32]>(&dp[0]));
+            tmem_ld_32x32(t_row + kColP + half * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&dp[32]));
             tmem_wait_ld();
-            uint32_t pk[16];
-            const int m = n_begin + n;
-            const int k_valid = subtile_ref(L, m).valid;
-            if (m >= 2 * i || k_valid < kSubTile) {
-                // masked sub-tiles: key x of sub-tile m is visible to query row r iff it is a valid row
-                // and, in the diagonal tile, 64 m + x <= 128 i + r
-                float ds[32];
-                int vis = k_valid - 1;
-                if (m >= 2 * i && row - (m & 1) * kSubTile < vis) vis = row - (m & 1) * kSubTile;
-                const int lim = vis - half * 32;  // visible iff e <= lim
+            tc_fence_before();
+            mbar_arrive(&bars->dp_free);
+            // Key x of the tile is visible to query row r iff it is one of the tile's valid rows and,
+            // in the diagonal tile, x <= r.  Off the diagonal a full tile needs no mask at all.
+            const int k_valid = tile_ref(L, j_begin + n).valid;
+            const bool last = (n == n_steps - 1);
+            const bool masked = last || k_valid < kTile;
+            const int vis = (last && row < k_valid) ? row : k_valid - 1;
+            const int lim = vis - half * 64;  // visible iff (column within this half) <= lim
+            const uint32_t tS = t_row + kColS + st * kTile + half * 64;
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, neg_lse2));
-                    if (e > lim) pe = 0.f;
-                    ds[e] = pe * (__uint_as_float(pr[e]) - Drow);
-                }
-                pack32(ds, pk);
-            } else {
-                // two columns per instruction for the multiply-adds
-                const uint64_t c2x2 = f2_pack(c2, c2), nlx2 = f2_pack(neg_lse2, neg_lse2), Dx2 = f2_pack(Drow, Drow);
+            for (int c = 0; c < 2; ++c) {
+                uint32_t sr[32];
+                tmem_ld_32x32(tS + c * 32, sr);
+                tmem_wait_ld();
+                uint32_t pk[16];
+                if (masked) {
 #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const uint64_t x = f2_fma(f2_pack(__uint_as_float(sr[2 * e]), __uint_as_float(sr[2 * e + 1])), c2x2, nlx2);
-                    float x0, x1;
-                    f2_unpack(x, x0, x1);
-                    const uint64_t pe = f2_pack(fast_exp2(x0), fast_exp2(x1));
-                    const uint64_t t = f2_sub(f2_pack(__uint_as_float(pr[2 * e]), __uint_as_float(pr[2 * e + 1])), Dx2);
-                    float d0, d1;
-                    f2_unpack(f2_mul(pe, t), d0, d1);
-                    pk[e] = pack_bf16(d0, d1);
+                    for (int e = 0; e < 16; ++e) {
+                        float pe0 = fast_exp2(fmaf(__uint_as_float(sr[2 * e]), c2, neg_lse2));
+                        float pe1 = fast_exp2(fmaf(__uint_as_float(sr[2 * e + 1]), c2, neg_lse2));
+                        if (c * 32 + 2 * e > lim) pe0 = 0.f;
+                        if (c * 32 + 2 * e + 1 > lim) pe1 = 0.f;
+                        pk[e] = pack_bf16(pe0 * (__uint_as_float(dp[c * 32 + 2 * e]) - Drow),
+                                          pe1 * (__uint_as_float(dp[c * 32 + 2 * e + 1]) - Drow));
+                    }
+                } else {
+                    // two columns per instruction for the multiply-adds
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const uint64_t x = f2_fma(f2_pack(__uint_as_float(sr[2 * e]), __uint_as_float(sr[2 * e + 1])), c2x2, nlx2);
+                        float x0, x1;
+                        f2_unpack(x, x0, x1);
+                        const uint64_t pe = f2_pack(fast_exp2(x0), fast_exp2(x1));
+                        const uint64_t t = f2_sub(f2_pack(__uint_as_float(dp[c * 32 + 2 * e]), __uint_as_float(dp[c * 32 + 2 * e + 1])), Dx2);
+                        float d0, d1;
+                        f2_unpack(f2_mul(pe, t), d0, d1);
+                        pk[e] = pack_bf16(d0, d1);
+                    }
                 }
+                // packed columns [16c, 16c+16) overlay score columns [16c, 16c+16) of this half, which
+                // have been read already (c = 1 writes over columns 16..31, read when c was 0)
+                tmem_st_32x16(tS + c * 16, pk);
             }
-            tmem_st_32x16(tS, pk);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(&bars->p_full[bf]);
+            mbar_arrive(&bars->p_full[st]);
         }
         if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDq + 6)) {
             tc_fence_after();
@@ -716,9 +783,9 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
 
 cudaError_t configure_bwd() {
     cudaError_t e;
-    e = cudaFuncSetAttribute(s2a_bwd_dq_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes);
+    e = cudaFuncSetAttribute(s2a_bwd_dq_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqCfg<64>::kSmemBytes);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(s2a_bwd_dq_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<128>::kSmemBytes);
+    e = cudaFuncSetAttribute(s2a_bwd_dq_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqCfg<128>::kSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(s2a_bwd_dkdv_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes);
     if (e != cudaSuccess) return e;
@@ -737,8 +804,8 @@ cudaError_t launch_bwd_preprocess(const PreParams& p, int d, cudaStream_t stream
 cudaError_t launch_bwd_dq(const BwdDqParams& p, int d, cudaStream_t stream) {
     const Geometry& g = p.geo;
     const unsigned grid = static_cast<unsigned>(static_cast<long long>(g.B) * g.H * g.groups * g.tiles_per_group);
-    if (d == 64) s2a_bwd_dq_kernel<64><<<grid, BwdCfg<64>::kThreads, BwdCfg<64>::kSmemBytes, stream>>>(p);
-    else s2a_bwd_dq_kernel<128><<<grid, BwdCfg<128>::kThreads, BwdCfg<128>::kSmemBytes, stream>>>(p);
+    if (d == 64) s2a_bwd_dq_kernel<64><<<grid, DqCfg<64>::kThreads, DqCfg<64>::kSmemBytes, stream>>>(p);
+    else s2a_bwd_dq_kernel<128><<<grid, DqCfg<128>::kThreads, DqCfg<128>::kSmemBytes, stream>>>(p);
     return cudaGetLastError();
 }
 

@@ -150,9 +150,9 @@ struct BwdBars {
 // for half the work and runs at 48 instead of 32 clocks per K step.
 //
 // Tensor memory columns: dQ [0,HD)   S buffers [128,256) [256,384)   dP [384,512)
-// Only one dP buffer fits, so the elementwise warps first copy their part of dP_n into registers and
-// release the buffer at once: dP_{n+1} (and S_{n+1}, into the other S buffer) run while they work on
-// step n.  Shared memory: Q_i and dO_i resident, a ring of three K tiles and a ring of two V tiles.
+// Only one dP buffer fits, so the elementwise warps copy their part of dP_{n+1} into registers as soon
+// as they are done with step n and release the buffer at once: dP_{n+2} (and S_{n+2}, into the S
+// buffer that the dQ MMAs of step n give back) run while they work on step n+1.  Shared memory: Q_i and dO_i resident, a ring of three K tiles and a ring of two V tiles.
 template <int HD>
 struct DqCfg {
     static constexpr int kThreads = 384;  // TMA warp, two MMA warps, one spare, 8 elementwise warps
@@ -175,7 +175,8 @@ struct DqBars {
     uint64_t acc_full;     // all dQ MMAs done
     uint64_t drain;        // abort path only (gradient MMA warp)
     uint64_t drain2;       // abort path only (score MMA warp)
-    uint64_t dp_full;      // S_n and dP_n are in tensor memory
+    uint64_t dp_ready;     // dP_n is in tensor memory
+    uint64_t s_ready[2];   // S_n is in tensor memory (buffer n & 1)
     uint64_t dp_free;      // every elementwise thread holds its part of dP_n in registers
     uint64_t p_full[2];    // bf16 dS_n is in tensor memory
     uint64_t buf_free[2];  // the dQ MMAs that read an S buffer's bf16 dS are done
@@ -227,9 +228,10 @@ __global__ void __launch_bounds__(DqCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(cons
         mbar_init(&bars->acc_full, 1);
         mbar_init(&bars->drain, 1);
         mbar_init(&bars->drain2, 1);
-        mbar_init(&bars->dp_full, 1);
+        mbar_init(&bars->dp_ready, 1);
         mbar_init(&bars->dp_free, 256);
         for (int x = 0; x < 2; ++x) {
+            mbar_init(&bars->s_ready[x], 1);
             mbar_init(&bars->p_full[x], 256);
             mbar_init(&bars->buf_free[x], 1);
             mbar_init(&bars->v_full[x], 1);
@@ -305,7 +307,11 @@ __global__ void __launch_bounds__(DqCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(cons
         for (int n = 0; ok && n < n_steps; ++n) {
             const int st = n & 1;
             const uint32_t ph = (n >> 1) & 1;
+            const int sk = n % C::kRingK;
+            // the two TMA barriers first: they have usually completed long ago, and every wait that sits
+            // between the two groups of MMAs below is time the tensor pipe idles
             if (!mbar_wait_uniform(&bars->v_full[st], ph, ctx, kWaitBwdDq + 2)) break;
+            if (!mbar_wait_uniform(&bars->k_full[sk], (n / C::kRingK) & 1, ctx, kWaitBwdDq + 10)) break;
             if (n >= 1 && !mbar_wait_uniform(&bars->dp_free, (n - 1) & 1, ctx, kWaitBwdDq + 9)) break;
             tc_fence_after();
             const uint32_t dV = desc_lo_k_major(smem_u32(sV + st * C::kTileBytes));
@@ -314,10 +320,9 @@ __global__ void __launch_bounds__(DqCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(cons
                 for (int kk = 0; kk < HD / 16; ++kk)
                     mma_ss(tP, dDO + desc_step_k_major(kk, C::kBoxBytes), dV + desc_step_k_major(kk, C::kBoxBytes), idesc_sc, kk > 0);
                 mma_commit(&bars->v_empty[st]);
+                mma_commit(&bars->dp_ready);
             }
             __syncwarp();
-            const int sk = n % C::kRingK;
-            if (!mbar_wait_uniform(&bars->k_full[sk], (n / C::kRingK) & 1, ctx, kWaitBwdDq + 10)) break;
             if (n >= 2 && !mbar_wait_uniform(&bars->buf_free[st], ph ^ 1, ctx, kWaitBwdDq + 7)) break;
             tc_fence_after();
             const uint32_t dK = desc_lo_k_major(smem_u32(sK + sk * C::kTileBytes));
@@ -326,7 +331,7 @@ __global__ void __launch_bounds__(DqCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(cons
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk)
                     mma_ss(tS, dQ + desc_step_k_major(kk, C::kBoxBytes), dK + desc_step_k_major(kk, C::kBoxBytes), idesc_sc, kk > 0);
-                mma_commit(&bars->dp_full);  // completes after every MMA issued so far: dP_n and S_n
+                mma_commit(&bars->s_ready[st]);
             }
             __syncwarp();
         }
@@ -386,16 +391,25 @@ __global__ void __launch_bounds__(DqCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(cons
         const float c2 = p.scale_log2;
         const uint64_t c2x2 = f2_pack(c2, c2), nlx2 = f2_pack(neg_lse2, neg_lse2), Dx2 = f2_pack(Drow, Drow);
         bool ok = true;
-        for (int n = 0; n < n_steps; ++n) {
-            const int st = n & 1;
-            if (!mbar_wait(&bars->dp_full, n & 1, ctx, kWaitBwdDq + 5)) { ok = false; break; }
+        uint32_t dp[64];  // this thread's part of dP_n
+        // Copy dP_m out of tensor memory and release its buffer.  Done for step 0 up front and for step
+        // n+1 at the END of step n (dP_{n+1} has been complete for a long time by then), so that dP_{n+2}
+        // and S_{n+2} can be issued while step n+1 is still being worked on.
+        auto fetch_dp = [&](int m) -> bool {
+            if (!mbar_wait(&bars->dp_ready, m & 1, ctx, kWaitBwdDq + 5)) return false;
             tc_fence_after();
-            uint32_t dp[64];
             tmem_ld_32x32(t_row + kColP + half * 64, *reinterpret_cast<uint32_t(*)[32]>(&dp[0]));
             tmem_ld_32x32(t_row + kColP + half * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&dp[32]));
             tmem_wait_ld();
             tc_fence_before();
             mbar_arrive(&bars->dp_free);
+            return true;
+        };
+        ok = fetch_dp(0);
+        for (int n = 0; ok && n < n_steps; ++n) {
+            const int st = n & 1;
+            if (!mbar_wait(&bars->s_ready[st], (n >> 1) & 1, ctx, kWaitBwdDq + 11)) { ok = false; break; }
+            tc_fence_after();
             // Key x of the tile is visible to query row r iff it is one of the tile's valid rows and,
             // in the diagonal tile, x <= r.  Off the diagonal a full tile needs no mask at all.
             const int k_valid = tile_ref(L, j_begin + n).valid;
@@ -441,6 +455,7 @@ __global__ void __launch_bounds__(DqCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(cons
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(&bars->p_full[st]);
+            if (n + 1 < n_steps && !fetch_dp(n + 1)) { ok = false; break; }
         }
         if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDq + 6)) {
             tc_fence_after();

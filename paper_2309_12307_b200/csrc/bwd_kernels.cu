@@ -131,9 +131,11 @@ struct BwdBars {
     uint64_t acc_full;            // all gradient MMAs done
     uint64_t drain;               // abort path only (gradient MMA warp)
     uint64_t drain2;              // abort path only (score MMA warp)
-    uint64_t s_full[3];           // score products of a step are in tensor memory
-    uint64_t p_full[3];           // bf16 P / dS of a step are in tensor memory
+    uint64_t s_full[3];           // S^T of a step is in tensor memory (buffer step % 3)
+    uint64_t p_full[3];           // bf16 P^T and dS^T of a step are in tensor memory
     uint64_t buf_free[3];         // gradient MMAs that read a score buffer's bf16 operands are done
+    uint64_t dp_ready;            // dP^T of a step is in tensor memory
+    uint64_t dp_free;             // every elementwise thread holds its part of dP^T in registers
     uint64_t st_full[kStages];    // streamed operands of a stage landed
     uint64_t st_empty[kStages];   // MMAs reading a stage are done
     uint32_t tmem_slot;
@@ -441,7 +443,8 @@ __global__ void __launch_bounds__(DqCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(cons
                         const uint64_t x = f2_fma(f2_pack(__uint_as_float(sr[2 * e]), __uint_as_float(sr[2 * e + 1])), c2x2, nlx2);
                         float x0, x1;
                         f2_unpack(x, x0, x1);
-                        const uint64_t pe = f2_pack(fast_exp2(x0), fast_exp2(x1));
+                        // part of the exponentials goes to the FMA pipe (see poly_exp2_x2)
+                        const uint64_t pe = ((kPolyExpMask >> e) & 1u) ? poly_exp2_x2(x) : f2_pack(fast_exp2(x0), fast_exp2(x1));
                         const uint64_t t = f2_sub(f2_pack(__uint_as_float(dp[c * 32 + 2 * e]), __uint_as_float(dp[c * 32 + 2 * e + 1])), Dx2);
                         float d0, d1;
                         f2_unpack(f2_mul(pe, t), d0, d1);
@@ -475,8 +478,12 @@ __global__ void __launch_bounds__(DqCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(cons
 // ------------------------------------------------------------------------------------------------
 // 3. dK, dV
 // ------------------------------------------------------------------------------------------------
-// Tensor memory columns: dV [0,HD)  dK [128,128+HD)  S^T buffers [256,320) [320,384)
-//                        dP^T buffers [384,448) [448,512)
+// Tensor memory columns: dV [0,HD)  dK [128,128+HD)  S^T buffers [256,320) [320,384) [384,448)
+//                        dP^T [448,512)
+// One dP^T buffer is enough because the elementwise warps copy their part of it into registers as soon
+// as they are done with the previous step (as in the dQ kernel); that leaves room for a third S^T
+// buffer, and with three steps in flight the chain scores -> elementwise -> gradient MMAs of one
+// buffer no longer leaves the tensor pipe idle.
 //
 // The CTA owns key tile (b, hk, original tokens tk0 .. tk0+127).  For every query head hq that
 // reads KV head hk (shift s): the tile sits at rolled position (tk0 - s) mod N, i.e. in group g at
@@ -503,6 +510,7 @@ template <int HD>
 __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(const __grid_constant__ BwdDkDvParams p) {
     using C = BwdCfg<HD>;
     using Bars = BwdBars<C::kStages>;
+    constexpr int kBufs = 3;  // S^T buffers in flight
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sK = smem;                                // resident: K_j
@@ -549,11 +557,13 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         mbar_init(&bars->acc_full, 1);
         mbar_init(&bars->drain, 1);
         mbar_init(&bars->drain2, 1);
-        for (int x = 0; x < 2; ++x) {
+        for (int x = 0; x < kBufs; ++x) {
             mbar_init(&bars->s_full[x], 1);
             mbar_init(&bars->p_full[x], 256);
             mbar_init(&bars->buf_free[x], 1);
         }
+        mbar_init(&bars->dp_ready, 1);
+        mbar_init(&bars->dp_free, 256);
         for (int st = 0; st < C::kStages; ++st) {
             mbar_init(&bars->st_full[st], 1);
             mbar_init(&bars->st_empty[st], 1);
@@ -574,7 +584,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_slot;
     const WaitCtx ctx{&bars->abort_flag, p.status};
-    constexpr uint32_t kColDV = 0, kColDK = 128, kColS = 256, kColP = 384;
+    constexpr uint32_t kColDV = 0, kColDK = 128, kColS = 256, kColP = 448;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -618,30 +628,38 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ---- score MMAs: S^T = K Q^T and dP^T = V dO^T of step `it` into buffer it & 1
+        // ---- score MMAs of step `it`: dP^T = V dO^T into the single dP^T buffer (free as soon as the
+        // elementwise warps hold the previous one in registers), then S^T = K Q^T into buffer it % 3
         // (warp-uniform loop, one elected lane issues; see the dQ kernel)
         constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);
         const uint32_t dK = desc_lo_k_major(smem_u32(sK)), dV = desc_lo_k_major(smem_u32(sV));
+        const uint32_t tP = tmem_base + kColP;
         bool ok = mbar_wait_uniform(&bars->res_full, 0, ctx, kWaitBwdDkDv + 3);
         for (int it = 0; ok && it < total_steps; ++it) {
             const int st = it % C::kStages;
+            const int bf = it % kBufs;
             if (!mbar_wait_uniform(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 2)) break;
-            if (it >= 2 && !mbar_wait_uniform(&bars->buf_free[it & 1], ((it - 2) >> 1) & 1, ctx, kWaitBwdDkDv + 8)) break;
+            if (it >= 1 && !mbar_wait_uniform(&bars->dp_free, (it - 1) & 1, ctx, kWaitBwdDkDv + 9)) break;
             tc_fence_after();
             const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
             const uint32_t dQ = desc_lo_k_major(aQ), dDO = desc_lo_k_major(aQ + C::kSubTileBytes);
-            const uint32_t tS = tmem_base + kColS + (it & 1) * kSubTile;
-            const uint32_t tP = tmem_base + kColP + (it & 1) * kSubTile;
+            if (elect_one()) {
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk)
+                    mma_ss(tP, dV + desc_step_k_major(kk, C::kBigBoxBytes), dDO + desc_step_k_major(kk, C::kSubBoxBytes),
+                           idesc_sc, kk > 0);
+                mma_commit(&bars->dp_ready);
+            }
+            __syncwarp();
+            if (it >= kBufs && !mbar_wait_uniform(&bars->buf_free[bf], ((it / kBufs) & 1) ^ 1, ctx, kWaitBwdDkDv + 8)) break;
+            tc_fence_after();
+            const uint32_t tS = tmem_base + kColS + bf * kSubTile;
             if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk)
                     mma_ss(tS, dK + desc_step_k_major(kk, C::kBigBoxBytes), dQ + desc_step_k_major(kk, C::kSubBoxBytes),
                            idesc_sc, kk > 0);
-#pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk)
-                    mma_ss(tP, dV + desc_step_k_major(kk, C::kBigBoxBytes), dDO + desc_step_k_major(kk, C::kSubBoxBytes),
-                           idesc_sc, kk > 0);
-                mma_commit(&bars->s_full[it & 1]);
+                mma_commit(&bars->s_full[bf]);
             }
             __syncwarp();
         }
@@ -653,17 +671,19 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         }
         __syncwarp();
     } else if (warp == 2) {
-        // ---- gradient MMAs: dV += P^T dO and dK += dS^T Q of step `it`
+        // ---- gradient MMAs: dV += P^T dO and dK += dS^T Q of step `it`; both bf16 operands sit in
+        // the step's S^T buffer (P^T in the first 16 packed columns of each thread's 32, dS^T in the rest)
         constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);
         for (int it = 0; it < total_steps; ++it) {
             const int st = it % C::kStages;
-            if (!mbar_wait_uniform(&bars->p_full[it & 1], (it >> 1) & 1, ctx, kWaitBwdDkDv + 4)) break;
+            const int bf = it % kBufs;
+            if (!mbar_wait_uniform(&bars->p_full[bf], (it / kBufs) & 1, ctx, kWaitBwdDkDv + 4)) break;
             tc_fence_after();
             const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
             const uint32_t dQmn = desc_lo_mn_major(aQ, C::kSubBoxBytes);
             const uint32_t dDOmn = desc_lo_mn_major(aQ + C::kSubTileBytes, C::kSubBoxBytes);
-            const uint32_t tPt = tmem_base + kColS + (it & 1) * kSubTile;   // bf16 P^T over the S^T buffer
-            const uint32_t tdSt = tmem_base + kColP + (it & 1) * kSubTile;  // bf16 dS^T over the dP^T buffer
+            const uint32_t tPt = tmem_base + kColS + bf * kSubTile;  // bf16 P^T
+            const uint32_t tdSt = tPt + 16;                          // bf16 dS^T
             if (elect_one()) {
 #pragma unroll
                 for (int kk = 0; kk < kSubTile / 16; ++kk)
@@ -674,7 +694,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                     mma_ts(tmem_base + kColDK, tdSt + packed_operand_col(kk), dQmn + kk * kDescStepMn, idesc_acc,
                            (it > 0) || (kk > 0));
                 mma_commit(&bars->st_empty[st]);
-                mma_commit(&bars->buf_free[it & 1]);
+                mma_commit(&bars->buf_free[bf]);
                 if (it == total_steps - 1) mma_commit(&bars->acc_full);
             }
             __syncwarp();
@@ -696,13 +716,27 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         const float c2 = p.scale_log2;
         bool ok = true;
         int it = 0;
+        uint32_t pr[32];  // this thread's part of dP^T of the current step
+        // Copy dP^T of step m out of tensor memory and release its buffer: for step 0 up front, for
+        // step m+1 at the end of step m (it has been complete for a long time by then).
+        auto fetch_dp = [&](int m) -> bool {
+            if (!mbar_wait(&bars->dp_ready, m & 1, ctx, kWaitBwdDkDv + 10)) return false;
+            tc_fence_after();
+            tmem_ld_32x32(t_row + kColP + half * 32, pr);
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(&bars->dp_free);
+            return true;
+        };
+        ok = fetch_dp(0);
         for (int hq = hq0; ok && hq < hq0 + rep; ++hq) {
             const HeadWalk w = head_walk(geo, hq, tk0);
             for (int n = w.n_begin; n < w.n_end; ++n, ++it) {
                 const int st = it % C::kStages;
+                const int bf = it % kBufs;
                 // the statistics of this step travel with its stage
                 if (!mbar_wait(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 5)) { ok = false; break; }
-                if (!mbar_wait(&bars->s_full[it & 1], (it >> 1) & 1, ctx, kWaitBwdDkDv + 6)) { ok = false; break; }
+                if (!mbar_wait(&bars->s_full[bf], (it / kBufs) & 1, ctx, kWaitBwdDkDv + 6)) { ok = false; break; }
                 tc_fence_after();
                 // lse[64] then D[64] of this stage; this thread's 32 columns start at float 32 * half.
                 // (explicit shared-memory loads: through a generic pointer they cost far more latency)
@@ -712,11 +746,11 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                     asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(a));
                     return r;
                 };
-                const uint32_t tS = t_row + kColS + (it & 1) * kSubTile + half * 32;
-                const uint32_t tP = t_row + kColP + (it & 1) * kSubTile + half * 32;
-                uint32_t sr[32], pr[32];
+                // this thread's 32 columns of S^T; its bf16 results go back over them once they are read:
+                // P^T into the first 16 (packed) columns, dS^T into the other 16
+                const uint32_t tS = t_row + kColS + bf * kSubTile + half * 32;
+                uint32_t sr[32];
                 tmem_ld_32x32(tS, sr);
-                tmem_ld_32x32(tP, pr);
                 tmem_wait_ld();
                 uint32_t pkP[16], pkS[16];
                 // query x of this sub-tile sees key row r iff x is a valid row of the sub-tile and, in the
@@ -771,10 +805,11 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                     }
                 }
                 tmem_st_32x16(tS, pkP);
-                tmem_st_32x16(tP, pkS);
+                tmem_st_32x16(tS + 16, pkS);
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(&bars->p_full[it & 1]);
+                mbar_arrive(&bars->p_full[bf]);
+                if (it + 1 < total_steps && !fetch_dp(it + 1)) { ok = false; break; }
             }
         }
         if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDkDv + 7)) {

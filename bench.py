@@ -33,7 +33,7 @@ FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_g
 # DRAM bytes (read + write) per launch from the ncu capture summarised in
 # profiles/dram_traffic_llama2_7b_8k.md, taken on llama2_7b_8k; every tensor is touched once, so
 # traffic scales with B*N*(H+Hkv)*d.  Set an entry to None when its kernel changes after the capture.
-NCU_TRAFFIC_8K = {"fwd": 249.4e6, "bwd_preprocess": 135.2e6, "bwd_dkdv": 373.5e6, "bwd_dq": 320.8e6}
+NCU_TRAFFIC_8K = {"fwd": 249.6e6, "bwd_preprocess": 137.9e6, "bwd_dkdv": 375.1e6, "bwd_dq": 322.8e6}
 NCU_TRAFFIC_8K_SIZE = 1 * 8192 * (32 + 32) * 128
 
 

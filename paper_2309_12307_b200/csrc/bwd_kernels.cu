@@ -480,8 +480,8 @@ __global__ void __launch_bounds__(DqCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(cons
 // ------------------------------------------------------------------------------------------------
 // Tensor memory columns: dV [0,HD)  dK [128,128+HD)  S^T buffers [256,320) [320,384) [384,448)
 //                        dP^T [448,512)
-// One dP^T buffer is enough because the elementwise warps copy their part of it into registers as soon
-// as they are done with the previous step (as in the dQ kernel); that leaves room for a third S^T
+// One dP^T buffer is enough because the elementwise warps copy their part of it into registers at the
+// start of a step and release the buffer at once; that leaves room for a third S^T
 // buffer, and with three steps in flight the chain scores -> elementwise -> gradient MMAs of one
 // buffer no longer leaves the tensor pipe idle.
 //
@@ -716,27 +716,25 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         const float c2 = p.scale_log2;
         bool ok = true;
         int it = 0;
-        uint32_t pr[32];  // this thread's part of dP^T of the current step
-        // Copy dP^T of step m out of tensor memory and release its buffer: for step 0 up front, for
-        // step m+1 at the end of step m (it has been complete for a long time by then).
-        auto fetch_dp = [&](int m) -> bool {
-            if (!mbar_wait(&bars->dp_ready, m & 1, ctx, kWaitBwdDkDv + 10)) return false;
-            tc_fence_after();
-            tmem_ld_32x32(t_row + kColP + half * 32, pr);
-            tmem_wait_ld();
-            tc_fence_before();
-            mbar_arrive(&bars->dp_free);
-            return true;
-        };
-        ok = fetch_dp(0);
         for (int hq = hq0; ok && hq < hq0 + rep; ++hq) {
             const HeadWalk w = head_walk(geo, hq, tk0);
             for (int n = w.n_begin; n < w.n_end; ++n, ++it) {
                 const int st = it % C::kStages;
                 const int bf = it % kBufs;
                 // the statistics of this step travel with its stage
-                if (!mbar_wait(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 5)) { ok = false; break; }
-                if (!mbar_wait(&bars->s_full[bf], (it / kBufs) & 1, ctx, kWaitBwdDkDv + 6)) { ok = false; break; }
+                // dP^T of this step has been complete for a long time: start copying this thread's part
+                // into registers, and release the single dP^T buffer as soon as the copy has landed, so
+                // that the dP^T product of the next step runs while this step is worked on
+                if (!mbar_wait(&bars->dp_ready, it & 1, ctx, kWaitBwdDkDv + 10)) { ok = false; break; }
+                tc_fence_after();
+                uint32_t pr[32];
+                tmem_ld_32x32(t_row + kColP + half * 32, pr);
+                if (!mbar_wait(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 5) ||
+                    !mbar_wait(&bars->s_full[bf], (it / kBufs) & 1, ctx, kWaitBwdDkDv + 6)) {
+                    tmem_wait_ld();  // giving up: let the copy that is in flight land first
+                    ok = false;
+                    break;
+                }
                 tc_fence_after();
                 // lse[64] then D[64] of this stage; this thread's 32 columns start at float 32 * half.
                 // (explicit shared-memory loads: through a generic pointer they cost far more latency)
@@ -752,6 +750,8 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                 uint32_t sr[32];
                 tmem_ld_32x32(tS, sr);
                 tmem_wait_ld();
+                tc_fence_before();
+                mbar_arrive(&bars->dp_free);
                 uint32_t pkP[16], pkS[16];
                 // query x of this sub-tile sees key row r iff x is a valid row of the sub-tile and, in the
                 // diagonal tile, 128 j + r <= 64 n + x
@@ -809,7 +809,6 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(&bars->p_full[bf]);
-                if (it + 1 < total_steps && !fetch_dp(it + 1)) { ok = false; break; }
             }
         }
         if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDkDv + 7)) {

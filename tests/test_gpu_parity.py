@@ -175,10 +175,11 @@ def test_leak_free_variant_matches_oracle(s2a):
     assert np.abs(o[:, : G // 2, H // 2:] - o_def[:, : G // 2, H // 2:]).max() > 1e-3
 
 
-def test_packed_qkv_equals_separate_tensors(s2a):
+@pytest.mark.parametrize("B,N,G,H,d", [(2, 1024, 512, 4, 128), (1, 1200, 200, 4, 64)])
+def test_packed_qkv_equals_separate_tensors(s2a, B, N, G, H, d):
     """Algorithm 1 takes qkv packed as [B, N, 3, H, d]; the packed entry points must give exactly
-    what the separate-tensor entry points give on the same values (only strides differ)."""
-    B, N, G, H, d = 2, 1024, 512, 4, 128
+    what the separate-tensor entry points give on the same values (only strides differ).  The
+    second shape has ragged tiles (G = 200)."""
     q, k, v, dO = (x.cuda() for x in make_inputs(B, N, H, H, d, seed=7))
     qkv = torch.stack([q, k, v], dim=2).contiguous()          # [B, N, 3, H, d]
     o, lse = s2a.s2a_fwd(q, k, v, G)

@@ -5,7 +5,7 @@
 //     dQ = scale * dS K    dK = scale * dS^T Q
 // Three kernels:
 //   1. preprocess: D[b,h,t] = sum_c dO[b,t,h,c] * o[b,t,h,c]                     (memory bound)
-//   2. dQ:   one CTA per 128-row query tile, streams 64-key sub-tiles of its group (keys <= query)
+//   2. dQ:   one CTA per 128-row query tile, walks the 128-key tiles of its group (keys <= query)
 //   3. dK,dV: one CTA per 128-row key tile, streams 64-query sub-tiles of every query head that
 //            shares the KV head (queries >= key), so the sum over those heads stays in tensor
 //            memory and needs no atomics.  It works on the transposed scores S^T = K Q^T so that
@@ -14,12 +14,15 @@
 // The roll of the shifted heads and the group boundaries are folded into TMA coordinates exactly
 // as in the forward kernel; all results are stored at original token rows.
 //
-// Both tensor-core kernels share one software pipeline (384 threads, one CTA per SM): warp 0
-// loads with TMA; warp 1 issues the score MMAs and warp 2 the gradient MMAs (a single issuing
-// warp spends so long on its own barrier waits that the tensor pipe runs dry in between; with two,
-// one can issue while the other waits); warps 4-11 do the elementwise work with one tensor-memory
-// lane and half of the columns per thread.  Score buffers are double-buffered, so the score
-// products of step n+1 run while the elementwise warps work on step n.
+// Both tensor-core kernels use the same software pipeline (384 threads, one CTA per SM, all 512
+// tensor-memory columns): warp 0 loads with TMA; warp 1 issues the score MMAs and warp 2 the
+// gradient MMAs (a single issuing warp spends so long on its own barrier waits that the tensor pipe
+// runs dry in between; with two, one can issue while the other waits); warp 3 owns the tensor-memory
+// allocation; warps 4-11 do the elementwise work with one tensor-memory lane and half of the columns
+// per thread.  dP (dP^T) has a single buffer: the elementwise warps copy their part of it into
+// registers and release it at once, which leaves the columns for two (dQ: 128 wide) or three (dK,dV:
+// 64 wide) score buffers, so that the score products of later steps run while the elementwise warps
+// work on the current one.
 #include "s2a_params.h"
 #include "sm100_ptx.cuh"
 

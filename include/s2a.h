@@ -165,11 +165,17 @@ int s2a_bwd_stage(const void* q, const void* k, const void* v, const void* o, co
                   void* workspace, size_t workspace_bytes, int stage, void* stream);
 
 /*
- * Forward + backward from HOST buffers (pinned memory recommended): copies q, k, v, dO to the
- * caller's device buffers, runs s2a_fwd and s2a_bwd, and copies o, lse, dq, dk, dv back, all
- * enqueued on `stream`; the caller synchronises the stream before reading the host outputs.
+ * Forward + backward from HOST buffers (pinned memory, or the copies are not asynchronous): q, k, v,
+ * dO go to the caller's device buffers, s2a_fwd and s2a_bwd run there, and o, lse, dq, dk, dv come
+ * back.  Heads are independent, so the work is cut into up to 8 chunks of whole KV heads and the
+ * copy of one chunk, the kernels of the previous one and the copy back of the one before that
+ * overlap (two copy streams owned by the library, created by the first call on a device, ordered
+ * against `stream` by events).  Everything is ordered after the work already in `stream` and
+ * `stream` is complete only when the last result has landed: the caller synchronises `stream`
+ * before reading the host outputs.  Results are bit-identical to s2a_fwd + s2a_bwd.
  *   h_*  : host pointers, same layouts and types as the device tensors
- *   d_*  : device buffers of the same sizes, owned by the caller (the library allocates nothing)
+ *   d_*  : device buffers of the same sizes, owned by the caller (the library allocates no memory);
+ *          used as staging space: their contents after the call are unspecified
  */
 int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const void* h_dO,
                      void* h_o, float* h_lse, void* h_dq, void* h_dk, void* h_dv,

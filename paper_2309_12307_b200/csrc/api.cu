@@ -19,9 +19,15 @@ __device__ int g_status_word;
 thread_local int tl_last_cuda_error = 0;
 
 constexpr int kMaxDevices = 64;
+constexpr int kMaxHostChunks = 8;
 struct DeviceState {
     bool ready = false;
     int* status_ptr = nullptr;
+    // s2a_fwd_bwd_host only: copy streams and the events that order them against the caller's stream
+    bool host_path_ready = false;
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_done = nullptr;
+    cudaEvent_t ev_in[kMaxHostChunks] = {}, ev_compute[kMaxHostChunks] = {};
 };
 DeviceState g_dev[kMaxDevices];
 
@@ -334,25 +340,75 @@ int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const vo
     int rc = check_shape(B, N, H, Hkv, d, G, 1.0f, H / 2, G / 2);
     if (rc != S2A_OK) return rc;
     if (!workspace || workspace_bytes < s2a_bwd_workspace_bytes(B, N, H, Hkv, d, G)) return S2A_ERR_INVALID_ARG;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t nq = static_cast<size_t>(B) * N * H * d * 2;
-    const size_t nk = static_cast<size_t>(B) * N * Hkv * d * 2;
-    const size_t nl = static_cast<size_t>(B) * H * N * sizeof(float);
+    DeviceState* ds = nullptr;
+    if ((rc = prepare_device(&ds)) != S2A_OK) return rc;
     cudaError_t e;
-    if ((e = cudaMemcpyAsync(d_q, h_q, nq, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaMemcpyAsync(d_k, h_k, nk, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaMemcpyAsync(d_v, h_v, nk, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaMemcpyAsync(d_dO, h_dO, nq, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
-    rc = s2a_fwd(d_q, d_k, d_v, d_o, d_lse, B, N, H, Hkv, d, G, stream);
-    if (rc != S2A_OK) return rc;
-    rc = s2a_bwd(d_q, d_k, d_v, d_o, d_lse, d_dO, d_dq, d_dk, d_dv, B, N, H, Hkv, d, G, workspace, workspace_bytes,
-                 stream);
-    if (rc != S2A_OK) return rc;
-    if ((e = cudaMemcpyAsync(h_o, d_o, nq, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaMemcpyAsync(h_lse, d_lse, nl, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaMemcpyAsync(h_dq, d_dq, nq, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaMemcpyAsync(h_dk, d_dk, nk, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaMemcpyAsync(h_dv, d_dv, nk, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+    if (!ds->host_path_ready) {
+        if ((e = cudaStreamCreateWithFlags(&ds->copy_in, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamCreateWithFlags(&ds->copy_out, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventCreateWithFlags(&ds->ev_start, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventCreateWithFlags(&ds->ev_done, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        for (int c = 0; c < kMaxHostChunks; ++c) {
+            if ((e = cudaEventCreateWithFlags(&ds->ev_in[c], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaEventCreateWithFlags(&ds->ev_compute[c], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        }
+        ds->host_path_ready = true;
+    }
+    // Heads are independent, so the job is cut into chunks of whole KV heads (with their query heads):
+    // while chunk c is computed, chunk c+1 travels to the device and the results of chunk c-1 travel
+    // back.  A chunk sits densely ([B, N, heads of the chunk, d]) in its share of the caller's buffers.
+    int chunks = 1;
+    for (int c = kMaxHostChunks; c > 1; c >>= 1) {
+        if (Hkv % c == 0) {
+            chunks = c;
+            break;
+        }
+    }
+    const int rep = H / Hkv;
+    const int kvc = Hkv / chunks, hc = kvc * rep;  // KV heads and query heads per chunk
+    const size_t rows = static_cast<size_t>(B) * N;
+    const size_t wq = static_cast<size_t>(hc) * d * 2, wk = static_cast<size_t>(kvc) * d * 2;  // bytes per token
+    const size_t pq = static_cast<size_t>(H) * d * 2, pk = static_cast<size_t>(Hkv) * d * 2;   // host pitches
+    const size_t wl = static_cast<size_t>(hc) * N * sizeof(float), pl = static_cast<size_t>(H) * N * sizeof(float);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    auto at = [](const void* base, size_t bytes) { return const_cast<char*>(static_cast<const char*>(base)) + bytes; };
+
+    if ((e = cudaEventRecord(ds->ev_start, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(ds->copy_in, ds->ev_start, 0)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(ds->copy_out, ds->ev_start, 0)) != cudaSuccess) return cuda_fail(e);
+    for (int c = 0; c < chunks; ++c) {
+        const size_t oq = c * rows * wq, ok_ = c * rows * wk, ol = static_cast<size_t>(c) * B * wl;
+        void *cq = at(d_q, oq), *ck = at(d_k, ok_), *cv = at(d_v, ok_), *cdo = at(d_dO, oq), *co = at(d_o, oq);
+        void *cdq = at(d_dq, oq), *cdk = at(d_dk, ok_), *cdv = at(d_dv, ok_);
+        float* cl = reinterpret_cast<float*>(at(d_lse, ol));
+        // host -> device: the chunk's heads of every token
+        if ((e = cudaMemcpy2DAsync(cq, wq, at(h_q, c * wq), pq, wq, rows, cudaMemcpyHostToDevice, ds->copy_in)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpy2DAsync(ck, wk, at(h_k, c * wk), pk, wk, rows, cudaMemcpyHostToDevice, ds->copy_in)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpy2DAsync(cv, wk, at(h_v, c * wk), pk, wk, rows, cudaMemcpyHostToDevice, ds->copy_in)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpy2DAsync(cdo, wq, at(h_dO, c * wq), pq, wq, rows, cudaMemcpyHostToDevice, ds->copy_in)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventRecord(ds->ev_in[c], ds->copy_in)) != cudaSuccess) return cuda_fail(e);
+        // compute on the caller's stream; the second half of ALL heads is shifted
+        if ((e = cudaStreamWaitEvent(st, ds->ev_in[c], 0)) != cudaSuccess) return cuda_fail(e);
+        int n_unshifted = H / 2 - c * hc;
+        n_unshifted = n_unshifted < 0 ? 0 : (n_unshifted > hc ? hc : n_unshifted);
+        const float scale = 1.0f / sqrtf(static_cast<float>(d));
+        rc = fwd_impl(cq, ck, cv, co, cl, B, N, hc, kvc, d, G, scale, n_unshifted, G / 2, 0u, stream, TokStrides());
+        if (rc != S2A_OK) return rc;
+        rc = bwd_impl(cq, ck, cv, co, cl, cdo, cdq, cdk, cdv, B, N, hc, kvc, d, G, scale, n_unshifted, G / 2, workspace,
+                      workspace_bytes, stream, kStageAll);
+        if (rc != S2A_OK) return rc;
+        if ((e = cudaEventRecord(ds->ev_compute[c], st)) != cudaSuccess) return cuda_fail(e);
+        // device -> host
+        if ((e = cudaStreamWaitEvent(ds->copy_out, ds->ev_compute[c], 0)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpy2DAsync(at(h_o, c * wq), pq, co, wq, wq, rows, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpy2DAsync(at(h_lse, c * wl), pl, cl, wl, wl, B, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpy2DAsync(at(h_dq, c * wq), pq, cdq, wq, wq, rows, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpy2DAsync(at(h_dk, c * wk), pk, cdk, wk, wk, rows, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpy2DAsync(at(h_dv, c * wk), pk, cdv, wk, wk, rows, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
+    }
+    // the caller's stream is done when the last copy back is
+    if ((e = cudaEventRecord(ds->ev_done, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(st, ds->ev_done, 0)) != cudaSuccess) return cuda_fail(e);
     return S2A_OK;
 }
 

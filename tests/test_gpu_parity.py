@@ -192,6 +192,31 @@ def test_packed_qkv_equals_separate_tensors(s2a, B, N, G, H, d):
     assert torch.equal(dqkv[:, :, 0], dq) and torch.equal(dqkv[:, :, 1], dk) and torch.equal(dqkv[:, :, 2], dv)
 
 
+@pytest.mark.parametrize("B,N,G,H,Hkv,d", [(1, 1024, 256, 4, 4, 64), (2, 1024, 512, 8, 2, 128), (1, 1200, 200, 4, 4, 64),
+                                           (1, 512, 256, 6, 3, 64)])
+def test_host_buffer_entry_point_equals_device_path(s2a, B, N, G, H, Hkv, d):
+    """s2a_fwd_bwd_host stages the heads through the device in chunks with its own copy streams; what
+    lands in the host outputs must be exactly what s2a_fwd + s2a_bwd give on device tensors, on
+    two calls in a row (the copy streams and events are reused)."""
+    q, k, v, dO = make_inputs(B, N, H, Hkv, d, seed=13)
+    dev = torch.device("cuda:0")
+    qd, kd, vd, dOd = (x.to(dev) for x in (q, k, v, dO))
+    o, lse = s2a.s2a_fwd(qd, kd, vd, G)
+    dq, dk, dv = s2a.s2a_bwd(qd, kd, vd, o, lse, dOd, G)
+    want = [x.cpu() for x in (o, lse, dq, dk, dv)]
+    pin = [x.pin_memory() for x in (q, k, v, dO)]
+    ws = torch.empty(max(s2a.bwd_workspace_bytes(B, N, H, Hkv, d, G), 256), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.Stream()
+    for _ in range(2):
+        host_out = [torch.full_like(x, float("nan")).pin_memory() for x in want]
+        dev_bufs = [torch.empty_like(x) for x in (qd, kd, vd, dOd, o, lse, dq, dk, dv)]
+        s2a.s2a_fwd_bwd_host(pin, host_out, dev_bufs, G, ws, stream=stream)
+        stream.synchronize()
+        assert s2a.device_status()[0] == 0
+        for got, ref in zip(host_out, want):
+            assert torch.equal(got, ref)
+
+
 def test_autograd_wrapper_matches_oracle(s2a):
     from paper_2309_12307_b200.autograd import s2_attn
 

@@ -156,6 +156,33 @@ def test_ragged_group_sizes_match_oracle_everywhere(s2a, B, N, G, H, Hkv, d, ex)
         assert rel_l2(dv[:, :, hk], dv_ref[:, :, hk]) <= GRAD_REL_L2, hk
 
 
+def test_many_small_units_sampled_rows(s2a):
+    """Batch 4 x 32 heads x 4 groups of a short sequence: 512 (batch, head, group) units, i.e. many more
+    units than SMs and several chunks of the block order; sampled rows against the oracle."""
+    B, N, G, H, Hkv, d = 4, 4096, 1024, 32, 8, 128
+    q, k, v, dO = make_inputs(B, N, H, Hkv, d, seed=21)
+    dev = torch.device("cuda:0")
+    qd, kd, vd, dOd = (x.to(dev) for x in (q, k, v, dO))
+    o, lse = s2a.s2a_fwd(qd, kd, vd, G)
+    dq, dk, dv = s2a.s2a_bwd(qd, kd, vd, o, lse, dOd, G)
+    torch.cuda.synchronize()
+    assert s2a.device_status()[0] == 0
+    rng = np.random.default_rng(3)
+    q_rows = [(int(b), int(h), int(t)) for b, h, t in zip(rng.integers(0, B, 40), rng.integers(0, H, 40), rng.integers(0, N, 40))]
+    q_rows += [(B - 1, H - 1, 0), (B - 1, H - 1, N - 1), (0, H // 2, G // 2), (B - 1, 0, N - 1)]
+    kv_rows = [(int(b), int(h), int(t)) for b, h, t in zip(rng.integers(0, B, 24), rng.integers(0, Hkv, 24), rng.integers(0, N, 24))]
+    o_ref, lse_ref = orc.fwd(q, k, v, G, rows=q_rows)
+    dq_ref, dk_ref, dv_ref = orc.bwd(q, k, v, dO, G, q_rows=q_rows, kv_rows=kv_rows)
+    qi = torch.tensor(q_rows, device=dev)
+    ki = torch.tensor(kv_rows, device=dev)
+    assert np.abs(o[qi[:, 0], qi[:, 2], qi[:, 1]].double().cpu().numpy() - o_ref).max() <= O_ATOL
+    assert np.abs(lse[qi[:, 0], qi[:, 1], qi[:, 2]].double().cpu().numpy() - lse_ref).max() <= LSE_ATOL
+    assert rel_l2(dq[qi[:, 0], qi[:, 2], qi[:, 1]].double().cpu().numpy(), dq_ref) <= GRAD_REL_L2
+    assert rel_l2(dk[ki[:, 0], ki[:, 2], ki[:, 1]].double().cpu().numpy(), dk_ref) <= GRAD_REL_L2
+    assert rel_l2(dv[ki[:, 0], ki[:, 2], ki[:, 1]].double().cpu().numpy(), dv_ref) <= GRAD_REL_L2
+    assert torch.isfinite(dq.float()).all() and torch.isfinite(dk.float()).all() and torch.isfinite(dv.float()).all()
+
+
 def test_leak_free_variant_matches_oracle(s2a):
     """Appendix B, variant 2 on a head-dim-128 GQA shape with eight tiles per group: the wrapped group
     of the shifted heads is cut at the wrap (tile 4 of 8)."""

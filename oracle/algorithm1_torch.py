@@ -46,11 +46,27 @@ def _group_causal_attention(q, k, v, scale, extra_mask=None):
     return out, lse
 
 
-def s2_attn(q, k, v, G, scale=None, leak_free=False):
+def _swap_halves_of_wrapped_group(x, B, n_groups, H):
+    """x: [B * n_groups, G, H, ...] in rolled, grouped order.  In the last group of every sequence
+    (the one that wraps) exchange the first and the second half of the tokens of heads H/2.. ;
+    applying it twice restores x."""
+    G = x.shape[1]
+    x = x.clone()
+    last = (torch.arange(B) * n_groups + (n_groups - 1)).tolist()
+    for bg in last:
+        blk = x[bg, :, H // 2:]
+        x[bg, :, H // 2:] = torch.cat([blk[G // 2:], blk[: G // 2]], dim=0)
+    return x
+
+
+def s2_attn(q, k, v, G, scale=None, leak_free=False, swap_wrapped=False):
     """q [B,N,H,d], k/v [B,N,Hkv,d] (fp64) -> o [B,N,H,d], lse [B,H,N].
     leak_free: variant 2 of Appendix B ("a small modification on the attention mask"): in the shifted
     heads the last group, which holds the sequence's last G/2 tokens followed by its first G/2 tokens,
-    is treated as two groups, so the front tokens do not attend the tail tokens."""
+    is treated as two groups, so the front tokens do not attend the tail tokens.
+    swap_wrapped: variant 3 of Appendix B ("swaps the shifted and the original front tokens"): in that same
+    group the two halves change places before the attention and change back after it, so the group is
+    attended in original token order (front tokens first)."""
     B, N, H, d = q.shape
     Hkv = k.shape[2]
     assert N % G == 0 and G % 2 == 0 and H % 2 == 0 and H % Hkv == 0
@@ -72,7 +88,13 @@ def s2_attn(q, k, v, G, scale=None, leak_free=False):
         # queries in the second half of that group (the front tokens) do not see its first half
         for bg in last.tolist():
             extra[bg, H // 2:, G // 2:, : G // 2] = True
+    if swap_wrapped:
+        assert not leak_free
+        q, k, v = (_swap_halves_of_wrapped_group(x, B, N // G, H) for x in (q, k, v))
     out, lse = _group_causal_attention(q, k, v, scale, extra)
+    if swap_wrapped:
+        out = _swap_halves_of_wrapped_group(out, B, N // G, H)
+        lse = _swap_halves_of_wrapped_group(lse.permute(0, 2, 1).unsqueeze(-1), B, N // G, H).squeeze(-1).permute(0, 2, 1)
     # step 4
     out = _roll_second_half(out.reshape(B, N, H, d), G // 2)
     lse = lse.reshape(B, N // G, H, G).permute(0, 2, 1, 3).reshape(B, H, N)  # rolled token order
@@ -80,11 +102,11 @@ def s2_attn(q, k, v, G, scale=None, leak_free=False):
     return out, lse.contiguous()
 
 
-def s2_attn_grads(q, k, v, dO, G, scale=None, leak_free=False):
+def s2_attn_grads(q, k, v, dO, G, scale=None, leak_free=False, swap_wrapped=False):
     """Autograd gradients of sum(o * dO) w.r.t. q, k, v (all fp64)."""
     q = q.detach().clone().requires_grad_(True)
     k = k.detach().clone().requires_grad_(True)
     v = v.detach().clone().requires_grad_(True)
-    o, _ = s2_attn(q, k, v, G, scale, leak_free)
+    o, _ = s2_attn(q, k, v, G, scale, leak_free, swap_wrapped)
     (o * dO).sum().backward()
     return q.grad, k.grad, v.grad

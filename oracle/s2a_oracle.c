@@ -67,7 +67,7 @@ typedef struct {
     int shift;       /* G/2 in the paper; sign = roll direction                 */
     int dtype;
     double scale;
-    int leak_free;   /* variant 2 of Appendix B: the wrapped tokens form a group of their own */
+    int variant;     /* 0 = Algorithm 1; 1 = variant 2 of Appendix B; 2 = variant 3 of Appendix B */
 } s2a_dims;
 
 static double bf16_to_f64(uint16_t bits) {
@@ -97,32 +97,66 @@ static int mod_n(long long x, int n) {
 static int head_shift(const s2a_dims* D, int h) { return h < D->n_unshifted ? 0 : D->shift; }
 
 /*
- * Variant 2 (Appendix B, "uses individual groups for the shifted tokens"): in a shifted head the
- * group that wraps around the sequence end -- it holds the last tokens of the sequence followed by
- * the first ones -- is cut in two at the wrap, so the front tokens no longer see the tail tokens.
- * pw is the rolled position of original token 0; the cut applies to the group containing it
- * (unless pw is a group boundary, where there is nothing to cut).
+ * Variants 2 and 3 of Appendix B concern the one group of a shifted head that wraps around the
+ * sequence end: it holds the last tokens of the sequence ("tail") followed by the first ones
+ * ("front"), so that in Algorithm 1 the front tokens attend the tail tokens.
+ *   variant 2 ("uses individual groups for the shifted tokens"): the group is cut in two at the wrap;
+ *             front tokens attend front tokens only, tail tokens attend tail tokens only.
+ *   variant 3 ("swaps the shifted and the original front tokens"): the two parts change places, so
+ *             the group is in original token order: front tokens come first (and attend only
+ *             themselves), tail tokens follow and attend all front tokens and the tail tokens before
+ *             them.
+ * pw is the rolled position of original token 0; the group containing it is the wrapped one (unless
+ * pw is a group boundary, where nothing wraps).
  */
 static int wrap_pos(const s2a_dims* D, int s) { return mod_n(-(long long)s, D->N); }
 
-/* first rolled position attended by the query at rolled position p (head with shift s) */
-static int first_attended(const s2a_dims* D, int s, int p) {
-    const int g_first = (p / D->G) * D->G;
-    if (D->leak_free && s != 0) {
-        const int pw = wrap_pos(D, s);
-        if (pw > g_first && pw <= p) return pw;
-    }
-    return g_first;
+/* up to two inclusive ranges of rolled positions, in the order in which the group is attended */
+typedef struct {
+    int n;
+    int lo[2], hi[2];
+} s2a_ranges;
+
+static int wrapped_at(const s2a_dims* D, int s, int g_first) {
+    if (s == 0) return -1;
+    const int pw = wrap_pos(D, s);
+    return (pw > g_first && pw < g_first + D->G) ? pw : -1;
 }
 
-/* one past the last rolled position whose query attends the key at rolled position pk */
-static int end_attending(const s2a_dims* D, int s, int pk) {
-    const int g_end = (pk / D->G + 1) * D->G;
-    if (D->leak_free && s != 0) {
-        const int pw = wrap_pos(D, s);
-        if (pw > pk && pw < g_end) return pw;
+/* keys attended by the query at rolled position p (head with shift s) */
+static s2a_ranges keys_of_query(const s2a_dims* D, int s, int p) {
+    s2a_ranges r;
+    const int g_first = (p / D->G) * D->G;
+    const int pw = D->variant ? wrapped_at(D, s, g_first) : -1;
+    r.n = 1, r.lo[0] = g_first, r.hi[0] = p;
+    if (pw >= 0) {
+        if (p >= pw) {
+            r.lo[0] = pw; /* a front token: front tokens up to itself, in both variants */
+        } else if (D->variant == 2) {
+            r.n = 2; /* a tail token after the swap: every front token, then the tail up to itself */
+            r.lo[0] = pw, r.hi[0] = g_first + D->G - 1;
+            r.lo[1] = g_first, r.hi[1] = p;
+        }
     }
-    return g_end;
+    return r;
+}
+
+/* queries that attend the key at rolled position pk */
+static s2a_ranges queries_of_key(const s2a_dims* D, int s, int pk) {
+    s2a_ranges r;
+    const int g_first = (pk / D->G) * D->G;
+    const int g_last = g_first + D->G - 1;
+    const int pw = D->variant ? wrapped_at(D, s, g_first) : -1;
+    r.n = 1, r.lo[0] = pk, r.hi[0] = g_last;
+    if (pw >= 0) {
+        if (pk < pw) {
+            r.hi[0] = pw - 1; /* a tail key: the tail tokens from itself on, in both variants */
+        } else if (D->variant == 2) {
+            r.n = 2; /* a front key after the swap: the front tokens from itself on, then every tail token */
+            r.lo[1] = g_first, r.hi[1] = pw - 1;
+        }
+    }
+    return r;
 }
 
 static size_t q_off(const s2a_dims* D, int b, int t, int h) {
@@ -147,27 +181,32 @@ static double fwd_row(const s2a_dims* D, const void* q, const void* k, const voi
     const int s = head_shift(D, h);
     const int hk = h / (D->H / D->Hkv);
     const int p = mod_n((long long)t - s, D->N);
-    const int p_first = first_attended(D, s, p);
-    const int n_att = p - p_first + 1;
+    const s2a_ranges att = keys_of_query(D, s, p);
+    int n_att = 0;
 
     load_row(q, q_off(D, b, t, h), D->d, D->dtype, qrow);
     double zmax = -INFINITY;
-    for (int i = 0; i < n_att; ++i) {
-        const int tk = mod_n((long long)p_first + i + s, D->N);
-        load_row(k, kv_off(D, b, tk, hk), D->d, D->dtype, krow);
-        zbuf[i] = D->scale * dot(qrow, krow, D->d);
-        if (zbuf[i] > zmax) zmax = zbuf[i];
+    for (int a = 0; a < att.n; ++a) {
+        for (int pp = att.lo[a]; pp <= att.hi[a]; ++pp, ++n_att) {
+            const int tk = mod_n((long long)pp + s, D->N);
+            load_row(k, kv_off(D, b, tk, hk), D->d, D->dtype, krow);
+            zbuf[n_att] = D->scale * dot(qrow, krow, D->d);
+            if (zbuf[n_att] > zmax) zmax = zbuf[n_att];
+        }
     }
     double sum = 0.0;
     for (int i = 0; i < n_att; ++i) sum += exp(zbuf[i] - zmax);
     const double lse = zmax + log(sum);
     if (o_row) {
         for (int c = 0; c < D->d; ++c) o_row[c] = 0.0;
-        for (int i = 0; i < n_att; ++i) {
-            const int tk = mod_n((long long)p_first + i + s, D->N);
-            const double w = exp(zbuf[i] - lse);
-            load_row(v, kv_off(D, b, tk, hk), D->d, D->dtype, krow);
-            for (int c = 0; c < D->d; ++c) o_row[c] += w * krow[c];
+        int i = 0;
+        for (int a = 0; a < att.n; ++a) {
+            for (int pp = att.lo[a]; pp <= att.hi[a]; ++pp, ++i) {
+                const int tk = mod_n((long long)pp + s, D->N);
+                const double w = exp(zbuf[i] - lse);
+                load_row(v, kv_off(D, b, tk, hk), D->d, D->dtype, krow);
+                for (int c = 0; c < D->d; ++c) o_row[c] += w * krow[c];
+            }
         }
     }
     return lse;
@@ -187,9 +226,9 @@ static int check_dims(const s2a_dims* D) {
  * rows != NULL: n_rows triples (b,h,t); o is [n_rows,d], lse is [n_rows].
  */
 int s2a_oracle_fwd_ex(const void* q, const void* k, const void* v, int dtype, int B, int N, int H, int Hkv, int d,
-                      int G, double scale, int n_unshifted, int shift, int leak_free, const int* rows,
+                      int G, double scale, int n_unshifted, int shift, int variant, const int* rows,
                       long long n_rows, double* o, double* lse) {
-    s2a_dims D = {B, N, H, Hkv, d, G, n_unshifted, shift, dtype, scale, leak_free};
+    s2a_dims D = {B, N, H, Hkv, d, G, n_unshifted, shift, dtype, scale, variant};
     if (check_dims(&D)) return -1;
     const long long total = rows ? n_rows : (long long)B * H * N;
     int err = 0;
@@ -240,10 +279,10 @@ int s2a_oracle_fwd(const void* q, const void* k, const void* v, int dtype, int B
  * summed on its own from the definition.
  */
 int s2a_oracle_bwd_ex(const void* q, const void* k, const void* v, const void* dO, int dtype, int B, int N, int H,
-                      int Hkv, int d, int G, double scale, int n_unshifted, int shift, int leak_free,
+                      int Hkv, int d, int G, double scale, int n_unshifted, int shift, int variant,
                       const int* q_rows, long long n_q, const int* kv_rows, long long n_kv, double* dq, double* dk,
                       double* dv) {
-    s2a_dims D = {B, N, H, Hkv, d, G, n_unshifted, shift, dtype, scale, leak_free};
+    s2a_dims D = {B, N, H, Hkv, d, G, n_unshifted, shift, dtype, scale, variant};
     if (check_dims(&D)) return -1;
     const int r = H / Hkv;
     const size_t n_stat = (size_t)B * H * N;
@@ -272,8 +311,9 @@ int s2a_oracle_bwd_ex(const void* q, const void* k, const void* v, const void* d
             for (int h = hk * r; h < (hk + 1) * r; ++h) {
                 const int s = head_shift(&D, h);
                 const int pk = mod_n((long long)tk - s, N);
-                const int g_end = end_attending(&D, s, pk); /* queries at rolled positions pk .. g_end-1 attend tk */
-                for (int p = pk; p < g_end; ++p) need[((size_t)b * H + h) * N + mod_n((long long)p + s, N)] = 1;
+                const s2a_ranges qs = queries_of_key(&D, s, pk); /* the queries that attend tk */
+                for (int a = 0; a < qs.n; ++a)
+                    for (int p = qs.lo[a]; p <= qs.hi[a]; ++p) need[((size_t)b * H + h) * N + mod_n((long long)p + s, N)] = 1;
             }
         }
     }
@@ -320,18 +360,20 @@ int s2a_oracle_bwd_ex(const void* q, const void* k, const void* v, const void* d
                 const int s = head_shift(&D, h);
                 const int hk = h / r;
                 const int p = mod_n((long long)t - s, N);
-                const int p_first = first_attended(&D, s, p);
+                const s2a_ranges att = keys_of_query(&D, s, p);
                 double* out = q_rows ? dq + (size_t)i * d : dq + q_off(&D, b, t, h);
                 for (int c = 0; c < d; ++c) out[c] = 0.0;
                 load_row(q, q_off(&D, b, t, h), d, dtype, qrow);
                 load_row(dO, q_off(&D, b, t, h), d, dtype, dorow);
-                for (int pp = p_first; pp <= p; ++pp) {
-                    const int tk = mod_n((long long)pp + s, N);
-                    load_row(k, kv_off(&D, b, tk, hk), d, dtype, krow);
-                    load_row(v, kv_off(&D, b, tk, hk), d, dtype, vrow);
-                    const double P = exp(scale * dot(qrow, krow, d) - lse[si]);
-                    const double dS = P * (dot(dorow, vrow, d) - Dsum[si]);
-                    for (int c = 0; c < d; ++c) out[c] += scale * dS * krow[c];
+                for (int a = 0; a < att.n; ++a) {
+                    for (int pp = att.lo[a]; pp <= att.hi[a]; ++pp) {
+                        const int tk = mod_n((long long)pp + s, N);
+                        load_row(k, kv_off(&D, b, tk, hk), d, dtype, krow);
+                        load_row(v, kv_off(&D, b, tk, hk), d, dtype, vrow);
+                        const double P = exp(scale * dot(qrow, krow, d) - lse[si]);
+                        const double dS = P * (dot(dorow, vrow, d) - Dsum[si]);
+                        for (int c = 0; c < d; ++c) out[c] += scale * dS * krow[c];
+                    }
                 }
             }
 
@@ -354,17 +396,19 @@ int s2a_oracle_bwd_ex(const void* q, const void* k, const void* v, const void* d
                 for (int h = hk * r; h < (hk + 1) * r; ++h) {
                     const int s = head_shift(&D, h);
                     const int pk = mod_n((long long)tk - s, N);
-                    const int g_end = end_attending(&D, s, pk);
-                    for (int p = pk; p < g_end; ++p) {
-                        const int t = mod_n((long long)p + s, N);
-                        const size_t si = ((size_t)b * H + h) * N + t;
-                        load_row(q, q_off(&D, b, t, h), d, dtype, qrow);
-                        load_row(dO, q_off(&D, b, t, h), d, dtype, dorow);
-                        const double P = exp(scale * dot(qrow, krow, d) - lse[si]);
-                        const double dS = P * (dot(dorow, vrow, d) - Dsum[si]);
-                        for (int c = 0; c < d; ++c) {
-                            out_v[c] += P * dorow[c];
-                            out_k[c] += scale * dS * qrow[c];
+                    const s2a_ranges qs = queries_of_key(&D, s, pk);
+                    for (int a = 0; a < qs.n; ++a) {
+                        for (int p = qs.lo[a]; p <= qs.hi[a]; ++p) {
+                            const int t = mod_n((long long)p + s, N);
+                            const size_t si = ((size_t)b * H + h) * N + t;
+                            load_row(q, q_off(&D, b, t, h), d, dtype, qrow);
+                            load_row(dO, q_off(&D, b, t, h), d, dtype, dorow);
+                            const double P = exp(scale * dot(qrow, krow, d) - lse[si]);
+                            const double dS = P * (dot(dorow, vrow, d) - Dsum[si]);
+                            for (int c = 0; c < d; ++c) {
+                                out_v[c] += P * dorow[c];
+                                out_k[c] += scale * dS * qrow[c];
+                            }
                         }
                     }
                 }

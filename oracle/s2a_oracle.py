@@ -90,9 +90,17 @@ def _defaults(H, G, d, scale, n_unshifted, shift):
     return float(scale), int(n_unshifted), int(shift)
 
 
-def fwd(q, k, v, G, scale=None, rows=None, n_unshifted=None, shift=None, leak_free=False):
+def _variant(leak_free, swap_wrapped) -> int:
+    """0 = Algorithm 1, 1 = variant 2 of Appendix B, 2 = variant 3 (they exclude each other)."""
+    if leak_free and swap_wrapped:
+        raise ValueError("variants 2 and 3 exclude each other")
+    return 1 if leak_free else (2 if swap_wrapped else 0)
+
+
+def fwd(q, k, v, G, scale=None, rows=None, n_unshifted=None, shift=None, leak_free=False, swap_wrapped=False):
     """o, lse.  rows=None: o [B,N,H,d], lse [B,H,N].  rows=[(b,h,t),...]: o [n,d], lse [n].
-    leak_free=True is variant 2 of Appendix B: the wrapped group of a shifted head is cut at the wrap."""
+    leak_free=True is variant 2 of Appendix B: the wrapped group of a shifted head is cut at the wrap.
+    swap_wrapped=True is variant 3: the two parts of the wrapped group change places (original token order)."""
     B, N, H, d = q.shape
     Hkv = k.shape[2]
     scale, n_unshifted, shift = _defaults(H, G, d, scale, n_unshifted, shift)
@@ -107,14 +115,15 @@ def fwd(q, k, v, G, scale=None, rows=None, n_unshifted=None, shift=None, leak_fr
     else:
         o = np.empty((n, d), dtype=np.float64)
         lse = np.empty((n,), dtype=np.float64)
-    rc = _load().s2a_oracle_fwd_ex(qp, kp, vp, dt, B, N, H, Hkv, d, G, scale, n_unshifted, shift, int(leak_free), rp, n,
+    rc = _load().s2a_oracle_fwd_ex(qp, kp, vp, dt, B, N, H, Hkv, d, G, scale, n_unshifted, shift, _variant(leak_free, swap_wrapped), rp, n,
                                    o.ctypes.data, lse.ctypes.data)
     if rc:
         raise ValueError(f"s2a_oracle_fwd_ex failed ({rc})")
     return o, lse
 
 
-def bwd(q, k, v, dO, G, scale=None, q_rows=None, kv_rows=None, n_unshifted=None, shift=None, leak_free=False):
+def bwd(q, k, v, dO, G, scale=None, q_rows=None, kv_rows=None, n_unshifted=None, shift=None, leak_free=False,
+        swap_wrapped=False):
     """dq, dk, dv.  With row lists: dq [n_q,d] for (b,h,t) rows, dk/dv [n_kv,d] for (b,hkv,t) rows."""
     B, N, H, d = q.shape
     Hkv = k.shape[2]
@@ -135,7 +144,7 @@ def bwd(q, k, v, dO, G, scale=None, q_rows=None, kv_rows=None, n_unshifted=None,
         qrp = dummy.ctypes.data
     if kv_rows is not None and nkv == 0:
         krp = dummy.ctypes.data
-    rc = _load().s2a_oracle_bwd_ex(qp, kp, vp, dp, dt, B, N, H, Hkv, d, G, scale, n_unshifted, shift, int(leak_free),
+    rc = _load().s2a_oracle_bwd_ex(qp, kp, vp, dp, dt, B, N, H, Hkv, d, G, scale, n_unshifted, shift, _variant(leak_free, swap_wrapped),
                                    qrp, nq,
                                    krp, nkv, dq.ctypes.data, dk.ctypes.data, dv.ctypes.data)
     if rc:

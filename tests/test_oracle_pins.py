@@ -443,3 +443,73 @@ def test_leak_free_variant_removes_exactly_the_leak():
         lp = (orc.fwd(*args_p, G, leak_free=True)[0] * dO.numpy()).sum()
         lm = (orc.fwd(*args_m, G, leak_free=True)[0] * dO.numpy()).sum()
         assert abs((lp - lm) / (2 * eps) - grad[idx]) < 1e-6
+
+
+# --------------------------------------------------------------------------- variant 3 (Appendix B)
+@pytest.mark.parametrize("B,N,G,H,Hkv,d", [(1, 16, 8, 2, 2, 4), (2, 32, 8, 4, 2, 5), (1, 16, 16, 2, 1, 4)])
+def test_swapped_variant_equals_swapped_transcription(B, N, G, H, Hkv, d):
+    """Variant 3: the two halves of the wrapped group of the shifted heads change places.  Index form
+    against the Algorithm-1 transcription that really swaps the tokens (and swaps back), forward and
+    autograd backward."""
+    q, k, v, dO = make_inputs_f64(B, N, H, Hkv, d, seed=41)
+    o_ref, lse_ref = alg1.s2_attn(q, k, v, G, swap_wrapped=True)
+    dq_ref, dk_ref, dv_ref = alg1.s2_attn_grads(q, k, v, dO, G, swap_wrapped=True)
+    o, lse = orc.fwd(q, k, v, G, swap_wrapped=True)
+    dq, dk, dv = orc.bwd(q, k, v, dO, G, swap_wrapped=True)
+    np.testing.assert_allclose(o, o_ref.numpy(), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(lse, lse_ref.numpy(), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(dq, dq_ref.numpy(), rtol=0, atol=1e-11)
+    np.testing.assert_allclose(dk, dk_ref.numpy(), rtol=0, atol=1e-11)
+    np.testing.assert_allclose(dv, dv_ref.numpy(), rtol=0, atol=1e-11)
+
+
+def test_swapped_variant_is_causal_attention_in_original_token_order():
+    """With variant 3 the wrapped group of a shifted head is plain causal attention over its tokens
+    taken in original order: the first G/2 tokens of the sequence, then the last G/2.  So no token
+    attends a later one any more, and every other row equals the default method."""
+    B, N, G, H, Hkv, d = 1, 64, 16, 4, 4, 8
+    q, k, v, dO = make_inputs_f64(B, N, H, Hkv, d, seed=43)
+    o_def, _ = orc.fwd(q, k, v, G)
+    o_v3, lse_v3 = orc.fwd(q, k, v, G, swap_wrapped=True)
+    half = G // 2
+    members = list(range(0, half)) + list(range(N - half, N))
+    for h in range(H // 2, H):
+        o_ref, lse_ref = _full_causal_attention(q[0, members, h], k[0, members, h], v[0, members, h], 1 / math.sqrt(d))
+        np.testing.assert_allclose(o_v3[0, members, h], o_ref.numpy(), atol=1e-12)
+        np.testing.assert_allclose(lse_v3[0, h, members], lse_ref.numpy(), atol=1e-12)
+    # only the wrapped group of the shifted heads changes (token 0 attends itself alone either way? no:
+    # by default it attends the tail as well, so all G tokens of the group change)
+    changed = np.abs(o_v3 - o_def).max(axis=-1)[0] > 1e-12     # [N, H]
+    assert not changed[:, : H // 2].any()
+    assert not changed[half:N - half, H // 2:].any()
+    assert changed[members][:, H // 2:].all()
+    # causality in original order: perturbing token t changes no output before t (any head)
+    for t_pert in (3, N - 3):
+        k2, v2 = k.clone(), v.clone()
+        k2[0, t_pert] += 1.0
+        v2[0, t_pert] -= 1.0
+        o_pert, _ = orc.fwd(q, k2, v2, G, swap_wrapped=True)
+        assert np.abs(o_pert - o_v3)[0, :t_pert].max() == 0.0
+    # ... which the default method violates (the leak): token 1 of a shifted head sees token N-3
+    k2, v2 = k.clone(), v.clone()
+    k2[0, N - 3] += 1.0
+    o_pert, _ = orc.fwd(q, k2, v2, G)
+    assert np.abs(o_pert - o_def)[0, 1, H // 2:].max() > 0.0
+    # gradients: finite differences on one coordinate of each input
+    dq, dk, dv = orc.bwd(q, k, v, dO, G, swap_wrapped=True)
+    eps = 1e-6
+    for x, grad, idx in ((q, dq, (0, N - 2, 3, 1)), (k, dk, (0, 2, 3, 0)), (v, dv, (0, N - 5, 2, 5))):
+        xp, xm = x.clone(), x.clone()
+        xp[idx] += eps
+        xm[idx] -= eps
+        args_p = [xp if t is x else t for t in (q, k, v)]
+        args_m = [xm if t is x else t for t in (q, k, v)]
+        lp = (orc.fwd(*args_p, G, swap_wrapped=True)[0] * dO.numpy()).sum()
+        lm = (orc.fwd(*args_m, G, swap_wrapped=True)[0] * dO.numpy()).sum()
+        assert abs((lp - lm) / (2 * eps) - grad[idx]) < 1e-6
+
+
+def test_variants_2_and_3_exclude_each_other():
+    q, k, v, _ = make_inputs_f64(1, 16, 2, 2, 4, seed=1)
+    with pytest.raises(ValueError):
+        orc.fwd(q, k, v, 8, leak_free=True, swap_wrapped=True)

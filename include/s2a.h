@@ -92,9 +92,15 @@ size_t s2a_bwd_workspace_bytes(int B, int N, int H, int Hkv, int d, int G);
  * (pass 1/sqrt(d) for the standard choice).  H may be odd here.
  * flags: S2A_FLAG_LEAK_FREE selects variant 2 of Appendix B ("individual groups for the shifted
  * tokens"): in a shifted head the group that wraps around the sequence end is cut in two at the
- * wrap, so the sequence's first tokens no longer attend its last tokens.  Other bits must be 0.
+ * wrap, so the sequence's first tokens no longer attend its last tokens.
+ * S2A_FLAG_SWAP_WRAPPED selects variant 3 ("swaps the shifted and the original front tokens"; its
+ * figure is not in the paper's text, so this is a reading): in that same group the two parts change
+ * places, i.e. the group is attended in original token order - the first tokens of the sequence, then
+ * its last ones - so that no token attends a later one.  The two flags exclude each other; other bits
+ * must be 0.
  */
 #define S2A_FLAG_LEAK_FREE 1u
+#define S2A_FLAG_SWAP_WRAPPED 2u
 int s2a_fwd_ex(const void* q, const void* k, const void* v, void* o, float* lse,
                int B, int N, int H, int Hkv, int d, int G,
                float scale, int n_unshifted, int shift, unsigned flags, void* stream);

@@ -206,11 +206,18 @@ def s2a_bwd_stage(q, k, v, o, lse, dO, G, dq, dk, dv, workspace, stage, stream=N
 
 
 S2A_FLAG_LEAK_FREE = 1
+S2A_FLAG_SWAP_WRAPPED = 2
 
 
-def s2a_fwd_ex(q, k, v, G, scale=None, n_unshifted=None, shift=None, leak_free=False, o=None, lse=None, stream=None):
+def _flags(leak_free, swap_wrapped) -> int:
+    return (S2A_FLAG_LEAK_FREE if leak_free else 0) | (S2A_FLAG_SWAP_WRAPPED if swap_wrapped else 0)
+
+
+def s2a_fwd_ex(q, k, v, G, scale=None, n_unshifted=None, shift=None, leak_free=False, o=None, lse=None, stream=None,
+               swap_wrapped=False):
     """Generalised forward: heads [0, n_unshifted) unshifted, the rest rolled by -shift tokens;
-    leak_free=True cuts the wrapped group of the shifted heads at the wrap (Appendix B, variant 2)."""
+    leak_free=True cuts the wrapped group of the shifted heads at the wrap (Appendix B, variant 2);
+    swap_wrapped=True makes its two parts change places (variant 3)."""
     B, N, H, Hkv, d = _dims(q, k)
     scale = 1.0 / math.sqrt(d) if scale is None else scale
     n_unshifted = H // 2 if n_unshifted is None else n_unshifted
@@ -218,13 +225,13 @@ def s2a_fwd_ex(q, k, v, G, scale=None, n_unshifted=None, shift=None, leak_free=F
     o = torch.empty_like(q) if o is None else o
     lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if lse is None else lse
     rc = load().s2a_fwd_ex(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), B, N, H, Hkv, d, G,
-                           scale, n_unshifted, shift, S2A_FLAG_LEAK_FREE if leak_free else 0, _stream_ptr(stream))
+                           scale, n_unshifted, shift, _flags(leak_free, swap_wrapped), _stream_ptr(stream))
     _check(rc, "s2a_fwd_ex")
     return o, lse
 
 
 def s2a_bwd_ex(q, k, v, o, lse, dO, G, scale=None, n_unshifted=None, shift=None, leak_free=False, workspace=None,
-               stream=None, dq=None, dk=None, dv=None):
+               stream=None, dq=None, dk=None, dv=None, swap_wrapped=False):
     B, N, H, Hkv, d = _dims(q, k)
     scale = 1.0 / math.sqrt(d) if scale is None else scale
     n_unshifted = H // 2 if n_unshifted is None else n_unshifted
@@ -237,7 +244,7 @@ def s2a_bwd_ex(q, k, v, o, lse, dO, G, scale=None, n_unshifted=None, shift=None,
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
     rc = load().s2a_bwd_ex(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), dO.data_ptr(),
                            dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, N, H, Hkv, d, G, scale, n_unshifted, shift,
-                           S2A_FLAG_LEAK_FREE if leak_free else 0, workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
+                           _flags(leak_free, swap_wrapped), workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     _check(rc, "s2a_bwd_ex")
     return dq, dk, dv
 

@@ -93,6 +93,12 @@ int make_tmap(CUtensorMap* tm, const void* base, int d, int heads, int N, int B,
     return S2A_OK;
 }
 
+// variants 2 and 3 of Appendix B exclude each other; no other bits are defined
+bool flags_ok(unsigned flags) {
+    return (flags & ~static_cast<unsigned>(S2A_FLAG_LEAK_FREE | S2A_FLAG_SWAP_WRAPPED)) == 0 &&
+           flags != (S2A_FLAG_LEAK_FREE | S2A_FLAG_SWAP_WRAPPED);
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int check_shape(int B, int N, int H, int Hkv, int d, int G, float scale, int n_unshifted, int shift) {
@@ -121,13 +127,14 @@ int check_default_shape(int N, int H, int d, int G) {
     return S2A_OK;
 }
 
-Geometry make_geometry(int B, int N, int H, int Hkv, int G, int n_unshifted, int shift, int leak_free = 0) {
+Geometry make_geometry(int B, int N, int H, int Hkv, int G, int n_unshifted, int shift, unsigned flags = 0u) {
     Geometry g;
     g.B = B, g.N = N, g.H = H, g.Hkv = Hkv, g.G = G;
     g.n_unshifted = n_unshifted;
     g.shift = shift;
     g.groups = N / G;
-    g.leak_free = leak_free;
+    g.leak_free = (flags & S2A_FLAG_LEAK_FREE) ? 1 : 0;
+    g.swap_wrapped = (flags & S2A_FLAG_SWAP_WRAPPED) ? 1 : 0;
     // the grid has one slot per (unit, tile rank); groups with fewer tiles leave their last slots idle
     g.tiles_per_group = 0;
     const int shifts[2] = {0, shift};
@@ -175,7 +182,7 @@ struct TokStrides {
 
 int fwd_impl(const void* q, const void* k, const void* v, void* o, float* lse, int B, int N, int H, int Hkv, int d,
              int G, float scale, int n_unshifted, int shift, unsigned flags, void* stream, const TokStrides& ts) {
-    if (flags & ~static_cast<unsigned>(S2A_FLAG_LEAK_FREE)) return S2A_ERR_INVALID_ARG;
+    if (!flags_ok(flags)) return S2A_ERR_INVALID_ARG;
     if (!q || !k || !v || !o || !lse) return S2A_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return S2A_ERR_INVALID_ARG;
     int rc = check_shape(B, N, H, Hkv, d, G, scale, n_unshifted, shift);
@@ -192,7 +199,7 @@ int fwd_impl(const void* q, const void* k, const void* v, void* o, float* lse, i
     p.o = static_cast<__nv_bfloat16*>(o);
     p.lse = lse;
     p.status = ds->status_ptr;
-    p.geo = make_geometry(B, N, H, Hkv, G, n_unshifted, shift, (flags & S2A_FLAG_LEAK_FREE) ? 1 : 0);
+    p.geo = make_geometry(B, N, H, Hkv, G, n_unshifted, shift, flags);
     p.scale_log2 = scale * kLog2eHost;
     cudaError_t e = launch_fwd(p, d, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? S2A_OK : cuda_fail(e);
@@ -247,8 +254,8 @@ int bwd_impl(const void* q, const void* k, const void* v, const void* o, const f
     rc = prepare_device(&ds);
     if (rc != S2A_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (flags & ~static_cast<unsigned>(S2A_FLAG_LEAK_FREE)) return S2A_ERR_INVALID_ARG;
-    const Geometry geo = make_geometry(B, N, H, Hkv, G, n_unshifted, shift, (flags & S2A_FLAG_LEAK_FREE) ? 1 : 0);
+    if (!flags_ok(flags)) return S2A_ERR_INVALID_ARG;
+    const Geometry geo = make_geometry(B, N, H, Hkv, G, n_unshifted, shift, flags);
     float* Dsum = static_cast<float*>(workspace);
 
     BwdDqParams pq;

@@ -503,7 +503,9 @@ __device__ __forceinline__ HeadWalk head_walk(const Geometry& geo, int hq, int t
     const int pos = mod_pos(tk0 - s, geo.N);
     w.L = group_layout(geo, s, pos / geo.G);
     const int in_group = pos % geo.G;
-    w.j = in_group < w.L.lenA ? in_group / kTile : w.L.nA + (in_group - w.L.lenA) / kTile;
+    const int nB = w.L.nTiles - w.L.nA;
+    w.j = in_group < w.L.lenA ? (w.L.swapped ? nB : 0) + in_group / kTile
+                              : (w.L.swapped ? 0 : w.L.nA) + (in_group - w.L.lenA) / kTile;
     w.n_begin = 2 * w.j;
     w.n_end = 2 * end_query_tile(w.L, w.j);
     return w;

@@ -42,6 +42,7 @@ struct Geometry {
     int tiles_per_group;  // largest number of 128-token tiles any group has (G / 128 when G and shift are multiples of 128)
     int groups;           // N / G
     int leak_free;        // variant 2 of Appendix B: cut the wrapped group of a shifted head at the wrap
+    int swap_wrapped;     // variant 3 of Appendix B: the two runs of the wrapped group change places
 };
 
 // Where the tokens of one group live.  Group g of a head with shift s holds rolled positions
@@ -49,11 +50,13 @@ struct Geometry {
 // that wraps past token N-1, a second run [0, lenB).  Each run is cut into 128-token tiles from its own
 // start, so a tile is always a contiguous range of original tokens (one TMA box, no wrap inside a
 // tile) and only the last tile of a run can have fewer than 128 valid rows.  Tiles are numbered in
-// rolled (= causal) order: the nA tiles of the first run, then those of the second.
+// causal order: the nA tiles of the first run, then those of the second (the other way round in
+// variant 3 of Appendix B).
 struct GroupLayout {
     int a0, lenA, lenB;
     int nA, nTiles;
-    int cut;  // variant 2: tile index at which the wrapped group is cut in two (0 = no cut)
+    int cut;      // variant 2: tile index at which the wrapped group is cut in two (0 = no cut)
+    int swapped;  // variant 3: the tiles of the second run ([0, lenB), the front of the sequence) come first
 };
 __host__ __device__ inline GroupLayout group_layout(const Geometry& geo, int s, int g) {
     GroupLayout L;
@@ -67,6 +70,8 @@ __host__ __device__ inline GroupLayout group_layout(const Geometry& geo, int s, 
     // Variant 2: the second run starts at original token 0; queries there attend keys from the cut
     // on, keys before the cut are attended by queries before the cut only.
     L.cut = (geo.leak_free && L.lenB > 0) ? L.nA : 0;
+    // Variant 3: the wrapped group is attended in original token order, front tokens first.
+    L.swapped = (geo.swap_wrapped && L.lenB > 0) ? 1 : 0;
     return L;
 }
 struct TileRef {
@@ -75,12 +80,15 @@ struct TileRef {
 };
 __host__ __device__ inline TileRef tile_ref(const GroupLayout& L, int i) {
     TileRef t;
-    if (i < L.nA) {
-        t.tok0 = L.a0 + i * kTile;
-        t.valid = L.lenA - i * kTile;
+    const int nFirst = L.swapped ? L.nTiles - L.nA : L.nA;  // tiles of the run that comes first
+    const bool in_run_a = L.swapped ? (i >= nFirst) : (i < nFirst);
+    const int k = (i < nFirst) ? i : i - nFirst;             // tile within its run
+    if (in_run_a) {
+        t.tok0 = L.a0 + k * kTile;
+        t.valid = L.lenA - k * kTile;
     } else {
-        t.tok0 = (i - L.nA) * kTile;
-        t.valid = L.lenB - (i - L.nA) * kTile;
+        t.tok0 = k * kTile;
+        t.valid = L.lenB - k * kTile;
     }
     if (t.valid > kTile) t.valid = kTile;
     return t;

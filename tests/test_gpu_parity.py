@@ -92,6 +92,9 @@ def test_generalised_shift_and_head_split(s2a):
         dict(leak_free=True),                               # Appendix B, variant 2
         dict(n_unshifted=1, shift=128, leak_free=True),
         dict(n_unshifted=2, shift=-(G // 2), leak_free=True),
+        dict(swap_wrapped=True),                            # Appendix B, variant 3
+        dict(n_unshifted=1, shift=128, swap_wrapped=True),
+        dict(n_unshifted=2, shift=-(G // 2), swap_wrapped=True),
     ]
     for ex in cases:
         o, lse, dq, dk, dv = run_gpu(s2a, q, k, v, dO, G, **ex)
@@ -120,6 +123,8 @@ RAGGED = [
     (1, 1200, 600, 4, 2, 64, dict(n_unshifted=2, shift=44, scale=0.3)),         # arbitrary shift (multiple of 4)
     (1, 1200, 600, 4, 2, 64, dict(n_unshifted=2, shift=44, leak_free=True)),
     (1, 904, 904, 2, 2, 64, dict(n_unshifted=2, shift=0)),                      # full causal attention, ragged length
+    (1, 3000, 1000, 4, 4, 128, dict(swap_wrapped=True)),                        # variant 3 with ragged runs
+    (2, 1200, 600, 4, 2, 64, dict(n_unshifted=2, shift=44, swap_wrapped=True)),
 ]
 
 
@@ -242,6 +247,28 @@ def test_host_buffer_entry_point_equals_device_path(s2a, B, N, G, H, Hkv, d):
         assert s2a.device_status()[0] == 0
         for got, ref in zip(host_out, want):
             assert torch.equal(got, ref)
+
+
+def test_swapped_variant_matches_oracle(s2a):
+    """Appendix B, variant 3 on a head-dim-128 GQA shape with eight tiles per group: in the wrapped group
+    of the shifted heads the four tiles of the sequence's front come before the four of its tail; and the
+    two variant flags exclude each other."""
+    B, N, G, H, Hkv, d = 2, 2048, 1024, 4, 2, 128
+    q, k, v, dO = make_inputs(B, N, H, Hkv, d, seed=6)
+    o, lse, dq, dk, dv = run_gpu(s2a, q, k, v, dO, G, swap_wrapped=True)
+    o_ref, lse_ref = orc.fwd(q, k, v, G, swap_wrapped=True)
+    dq_ref, dk_ref, dv_ref = orc.bwd(q, k, v, dO, G, swap_wrapped=True)
+    assert np.abs(o - o_ref).max() <= O_ATOL
+    assert np.abs(lse - lse_ref).max() <= LSE_ATOL
+    for got, want in ((dq, dq_ref), (dk, dk_ref), (dv, dv_ref)):
+        assert rel_l2(got, want) <= GRAD_REL_L2
+    # it differs from the default method exactly in the wrapped group of the shifted heads
+    o_def, _ = orc.fwd(q, k, v, G)
+    assert np.abs(o_ref - o_def)[:, G // 2:N - G // 2].max() == 0.0
+    assert np.abs(o - o_def)[:, :G // 2, H // 2:].max() > 0.1
+    with pytest.raises(s2a.S2AError) as e:
+        s2a.s2a_fwd_ex(q.cuda(), k.cuda(), v.cuda(), G, leak_free=True, swap_wrapped=True)
+    assert e.value.status == s2a.S2A_ERR_INVALID_ARG
 
 
 def test_autograd_wrapper_matches_oracle(s2a):

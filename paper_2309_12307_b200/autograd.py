@@ -1,7 +1,7 @@
 """torch.autograd front end of S2-Attn (Algorithm 1 of the LongLoRA paper).
 
 `s2_attn(q, k, v, G)` behaves like a differentiable function of q [B,N,H,d] and k, v [B,N,Hkv,d]
-(bf16, CUDA, contiguous): the forward runs `s2a_fwd`, the backward `s2a_bwd`.  Everything is
+(bf16, CUDA, contiguous): the forward runs `s2a_fwd_ex`, the backward `s2a_bwd_ex`.  Everything is
 computed by the CUDA library; torch only records the graph and owns the tensors.
 """
 from __future__ import annotations
@@ -13,20 +13,28 @@ from . import binding
 
 class _S2Attn(torch.autograd.Function):
     @staticmethod
-    def forward(ctx, q, k, v, G):
+    def forward(ctx, q, k, v, G, opts):
         q, k, v = q.contiguous(), k.contiguous(), v.contiguous()
-        o, lse = binding.s2a_fwd(q, k, v, G)
+        o, lse = binding.s2a_fwd_ex(q, k, v, G, **opts)
         ctx.save_for_backward(q, k, v, o, lse)
-        ctx.G = G
+        ctx.G, ctx.opts = G, opts
         return o
 
     @staticmethod
     def backward(ctx, dO):
         q, k, v, o, lse = ctx.saved_tensors
-        dq, dk, dv = binding.s2a_bwd(q, k, v, o, lse, dO.contiguous(), ctx.G)
-        return dq, dk, dv, None
+        dq, dk, dv = binding.s2a_bwd_ex(q, k, v, o, lse, dO.contiguous(), ctx.G, **ctx.opts)
+        return dq, dk, dv, None, None
 
 
-def s2_attn(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, G: int) -> torch.Tensor:
-    """Shifted sparse attention: groups of G tokens, second half of the heads shifted by G/2."""
-    return _S2Attn.apply(q, k, v, G)
+def s2_attn(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, G: int, *, scale: float | None = None,
+            n_unshifted: int | None = None, shift: int | None = None, leak_free: bool = False,
+            swap_wrapped: bool = False) -> torch.Tensor:
+    """Shifted sparse attention: groups of G tokens, second half of the heads shifted by G/2.
+
+    Keyword options as in `s2a_fwd_ex`: softmax scale (default 1/sqrt(d)), number of unshifted heads
+    (default H/2), shift in tokens (default G/2), and variants 2 (`leak_free`) and 3 (`swap_wrapped`)
+    of the paper's Appendix B.  With n_unshifted = H, shift = 0 and G = N it is ordinary causal attention.
+    """
+    opts = dict(scale=scale, n_unshifted=n_unshifted, shift=shift, leak_free=leak_free, swap_wrapped=swap_wrapped)
+    return _S2Attn.apply(q, k, v, G, opts)

@@ -285,6 +285,17 @@ def test_autograd_wrapper_matches_oracle(s2a):
     assert np.abs(o.detach().double().cpu().numpy() - o_ref).max() <= O_ATOL
     for got, want in ((qd.grad, dq_ref), (kd.grad, dk_ref), (vd.grad, dv_ref)):
         assert rel_l2(got.double().cpu().numpy(), want) <= GRAD_REL_L2
+    # with options: variant 3 and a custom scale
+    ex = dict(swap_wrapped=True, scale=0.11)
+    qd, kd, vd = (x.cuda().requires_grad_(True) for x in (q, k, v))
+    o = s2_attn(qd, kd, vd, G, **ex)
+    (o.float() * dO.cuda().float()).sum().backward()
+    torch.cuda.synchronize()
+    o_ref, _ = orc.fwd(q, k, v, G, **ex)
+    dq_ref, dk_ref, dv_ref = orc.bwd(q, k, v, dO, G, **ex)
+    assert np.abs(o.detach().double().cpu().numpy() - o_ref).max() <= O_ATOL
+    for got, want in ((qd.grad, dq_ref), (kd.grad, dk_ref), (vd.grad, dv_ref)):
+        assert rel_l2(got.double().cpu().numpy(), want) <= GRAD_REL_L2
 
 
 def test_outputs_are_deterministic_and_fully_written(s2a):

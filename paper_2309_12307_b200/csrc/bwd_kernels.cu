@@ -137,7 +137,6 @@ struct BwdBars {
     uint64_t s_full[3];           // S^T of a step is in tensor memory (buffer step % 3)
     uint64_t p_full[3];           // bf16 P^T and dS^T of a step are in tensor memory
     uint64_t buf_free[3];         // gradient MMAs that read a score buffer's bf16 operands are done
-    uint64_t dp_ready;            // dP^T of a step is in tensor memory
     uint64_t dp_free;             // every elementwise thread holds its part of dP^T in registers
     uint64_t st_full[kStages];    // streamed operands of a stage landed
     uint64_t st_empty[kStages];   // MMAs reading a stage are done
@@ -567,7 +566,6 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
             mbar_init(&bars->p_full[x], 256);
             mbar_init(&bars->buf_free[x], 1);
         }
-        mbar_init(&bars->dp_ready, 1);
         mbar_init(&bars->dp_free, 256);
         for (int st = 0; st < C::kStages; ++st) {
             mbar_init(&bars->st_full[st], 1);
@@ -653,7 +651,6 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                 for (int kk = 0; kk < HD / 16; ++kk)
                     mma_ss(tP, dV + desc_step_k_major(kk, C::kBigBoxBytes), dDO + desc_step_k_major(kk, C::kSubBoxBytes),
                            idesc_sc, kk > 0);
-                mma_commit(&bars->dp_ready);
             }
             __syncwarp();
             if (it >= kBufs && !mbar_wait_uniform(&bars->buf_free[bf], ((it / kBufs) & 1) ^ 1, ctx, kWaitBwdDkDv + 8)) break;
@@ -727,20 +724,19 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                 const int st = it % C::kStages;
                 const int bf = it % kBufs;
                 // the statistics of this step travel with its stage
-                // dP^T of this step has been complete for a long time: start copying this thread's part
-                // into registers, and release the single dP^T buffer as soon as the copy has landed, so
-                // that the dP^T product of the next step runs while this step is worked on
-                if (!mbar_wait(&bars->dp_ready, it & 1, ctx, kWaitBwdDkDv + 10)) { ok = false; break; }
-                tc_fence_after();
-                uint32_t pr[32];
-                tmem_ld_32x32(t_row + kColP + half * 32, pr);
+                // s_full covers dP^T of this step as well: its MMAs were issued before those of S^T by the
+                // same thread, and a commit completes after everything issued before it
                 if (!mbar_wait(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 5) ||
                     !mbar_wait(&bars->s_full[bf], (it / kBufs) & 1, ctx, kWaitBwdDkDv + 6)) {
-                    tmem_wait_ld();  // giving up: let the copy that is in flight land first
                     ok = false;
                     break;
                 }
                 tc_fence_after();
+                // copy this thread's part of dP^T into registers and release the single dP^T buffer as
+                // soon as the copy has landed, so that the dP^T product of the next step runs while this
+                // step is worked on
+                uint32_t pr[32];
+                tmem_ld_32x32(t_row + kColP + half * 32, pr);
                 // lse[64] then D[64] of this stage; this thread's 32 columns start at float 32 * half.
                 // (explicit shared-memory loads: through a generic pointer they cost far more latency)
                 const uint32_t stat_sa = smem_u32(sStat + st * 2 * kSubTile) + half * 128;

@@ -33,6 +33,9 @@
  *     never approximated.
  *   - Rows of a partly masked tile that belong to a neighbouring group are read (and masked), so a
  *     NaN or infinity in one token's k or v can reach the outputs of the adjacent group's tokens.
+ *   - Host threads: entry points may be called from several host threads (the one-time set-up of a
+ *     device is serialised); s2a_fwd_bwd_host and s2a_bwd_noalloc keep per-device state (copy streams,
+ *     built-in scratch), so calls of either on one device must not overlap.
  *   - Device-side waits are bounded.  If one ever expires the kernel records where, stops cleanly,
  *     and s2a_device_status() reports it; outputs of that launch are then undefined.
  */

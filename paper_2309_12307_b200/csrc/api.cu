@@ -6,6 +6,8 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "../../include/s2a.h"
 #include "s2a_params.h"
 
@@ -30,6 +32,7 @@ struct DeviceState {
     cudaEvent_t ev_in[kMaxHostChunks] = {}, ev_compute[kMaxHostChunks] = {};
 };
 DeviceState g_dev[kMaxDevices];
+std::mutex g_dev_mutex;  // guards the one-time set-up of a DeviceState (calls may come from several host threads)
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -48,6 +51,7 @@ int prepare_device(DeviceState** out) {
     if (e != cudaSuccess) return cuda_fail(e);
     if (dev < 0 || dev >= kMaxDevices) return S2A_ERR_UNSUPPORTED;
     DeviceState& ds = g_dev[dev];
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
     if (!ds.ready) {
         int major = 0;
         e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
@@ -350,6 +354,7 @@ int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const vo
     DeviceState* ds = nullptr;
     if ((rc = prepare_device(&ds)) != S2A_OK) return rc;
     cudaError_t e;
+    std::unique_lock<std::mutex> lock(g_dev_mutex);
     if (!ds->host_path_ready) {
         if ((e = cudaStreamCreateWithFlags(&ds->copy_in, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
         if ((e = cudaStreamCreateWithFlags(&ds->copy_out, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
@@ -361,6 +366,7 @@ int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const vo
         }
         ds->host_path_ready = true;
     }
+    lock.unlock();
     // Heads are independent, so the job is cut into chunks of whole KV heads (with their query heads):
     // while chunk c is computed, chunk c+1 travels to the device and the results of chunk c-1 travel
     // back.  A chunk sits densely ([B, N, heads of the chunk, d]) in its share of the caller's buffers.
@@ -438,6 +444,7 @@ int builtin_scratch(float** out) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(e);
     if (dev < 0 || dev >= kMaxDevices) return S2A_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
     if (!g_builtin_scratch_ptr[dev]) {
         void* ptr = nullptr;
         e = cudaGetSymbolAddress(&ptr, g_builtin_scratch);

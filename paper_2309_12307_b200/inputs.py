@@ -78,6 +78,16 @@ def make_inputs(B: int, N: int, H: int, Hkv: int, d: int, seed: int = 0):
     return tuple(out)
 
 
+def make_inputs_periodic(B: int, N: int, H: int, Hkv: int, d: int, period: int, seed: int = 0):
+    """Like make_inputs, but only `period` tokens per sequence are drawn and then repeated along N
+    (N a multiple of `period`): a quick way to fill very large tensors, e.g. to exercise offsets
+    beyond 2^31 elements.  Every batch entry gets its own draw."""
+    assert N % period == 0
+    q, k, v, dO = make_inputs(B, period, H, Hkv, d, seed)
+    reps = N // period
+    return tuple(x.repeat(1, reps, 1, 1).contiguous() for x in (q, k, v, dO))
+
+
 def make_workload_inputs(w: Workload, seed: int = 0):
     return make_inputs(w.B, w.N, w.H, w.Hkv, w.d, seed)
 

@@ -11,7 +11,7 @@ import pytest
 import torch
 
 from oracle import s2a_oracle as orc
-from paper_2309_12307_b200.inputs import WORKLOADS, make_inputs
+from paper_2309_12307_b200.inputs import WORKLOADS, make_inputs, make_inputs_periodic
 
 pytestmark = pytest.mark.gpu
 
@@ -186,6 +186,41 @@ def test_many_small_units_sampled_rows(s2a):
     assert rel_l2(dk[ki[:, 0], ki[:, 2], ki[:, 1]].double().cpu().numpy(), dk_ref) <= GRAD_REL_L2
     assert rel_l2(dv[ki[:, 0], ki[:, 2], ki[:, 1]].double().cpu().numpy(), dv_ref) <= GRAD_REL_L2
     assert torch.isfinite(dq.float()).all() and torch.isfinite(dk.float()).all() and torch.isfinite(dv.float()).all()
+
+
+def test_tensors_of_more_than_2_31_elements(s2a):
+    """B * N * H * d = 2.18e9 elements per query-side tensor (4.4 GB): every offset into q, o, dO, dq is
+    computed in 64 bits or wrong.  Rows of the last batch entry, last group (the highest addresses), and of
+    the first, against the oracle."""
+    B, N, G, H, Hkv, d = 2, 266240, 66560, 32, 8, 128
+    assert B * N * H * d > 2 ** 31
+    q, k, v, dO = make_inputs_periodic(B, N, H, Hkv, d, period=4096, seed=17)
+    dev = torch.device("cuda:0")
+    qd, kd, vd, dOd = (x.to(dev) for x in (q, k, v, dO))
+    o, lse = s2a.s2a_fwd(qd, kd, vd, G)
+    dq, dk, dv = s2a.s2a_bwd(qd, kd, vd, o, lse, dOd, G)
+    torch.cuda.synchronize()
+    assert s2a.device_status()[0] == 0
+    q_rows = [(1, H - 1, N - 1), (1, H - 1, G // 2 - 1), (1, H // 2 - 1, N - 1), (1, 0, N - G + 5), (1, H - 1, N - G // 2 - 1),
+              (0, 0, 0), (0, H - 1, G // 2), (0, 3, 70000), (1, 17, 200001)]
+    # key rows near the end of their group in their head's partition (few queries attend them, so the
+    # oracle stays fast): KV head 0 is unshifted, KV head Hkv-1 serves shifted query heads only
+    kv_rows = [(1, 0, N - 2), (1, 0, N - 130), (0, 0, G - 1), (1, Hkv - 1, G // 2 - 3), (1, Hkv - 1, G + G // 2 - 70),
+               (1, Hkv - 1, N - G // 2 - 2)]
+    o_ref, lse_ref = orc.fwd(q, k, v, G, rows=q_rows)
+    dq_ref, dk_ref, dv_ref = orc.bwd(q, k, v, dO, G, q_rows=q_rows, kv_rows=kv_rows)
+    qi = torch.tensor(q_rows, device=dev)
+    ki = torch.tensor(kv_rows, device=dev)
+    assert np.abs(o[qi[:, 0], qi[:, 2], qi[:, 1]].double().cpu().numpy() - o_ref).max() <= O_ATOL
+    assert np.abs(lse[qi[:, 0], qi[:, 1], qi[:, 2]].double().cpu().numpy() - lse_ref).max() <= LSE_ATOL
+    assert rel_l2(dq[qi[:, 0], qi[:, 2], qi[:, 1]].double().cpu().numpy(), dq_ref) <= GRAD_REL_L2
+    assert rel_l2(dk[ki[:, 0], ki[:, 2], ki[:, 1]].double().cpu().numpy(), dk_ref) <= GRAD_REL_L2
+    assert rel_l2(dv[ki[:, 0], ki[:, 2], ki[:, 1]].double().cpu().numpy(), dv_ref) <= GRAD_REL_L2
+    # the first member of every group attends only itself: o = v there, in the last batch entry too
+    t_first = torch.tensor([(g * G + G // 2) % N for g in range(N // G)], device=dev)
+    assert torch.equal(o[1, t_first, H - 1], vd[1, t_first, Hkv - 1])
+    del qd, kd, vd, dOd, o, lse, dq, dk, dv
+    torch.cuda.empty_cache()
 
 
 def test_leak_free_variant_matches_oracle(s2a):

@@ -30,9 +30,9 @@ METRIC = "S2-Attn fwd+bwd TFLOP/s (causal in-group FLOPs)"
 UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "llama2_7b_32k"
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
-# DRAM bytes (read + write) per launch from the ncu capture summarised in
-# profiles/dram_traffic_llama2_7b_8k.md, taken on llama2_7b_8k; every tensor is touched once, so
-# traffic scales with B*N*(H+Hkv)*d.  Set an entry to None when its kernel changes after the capture.
+# DRAM bytes (read + write) per launch, from one ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum) of each kernel on llama2_7b_8k; every tensor is touched once, so traffic
+# scales with B*N*(H+Hkv)*d.  An entry is None once its kernel has changed since the capture.
 NCU_TRAFFIC_8K = {"fwd": 249.6e6, "bwd_preprocess": 137.9e6, "bwd_dkdv": 375.1e6, "bwd_dq": 322.8e6}
 NCU_TRAFFIC_8K_SIZE = 1 * 8192 * (32 + 32) * 128
 
@@ -144,27 +144,74 @@ def oracle_sample_flops(w, n: int) -> float:
     return rep * w.d * (4.0 * pairs_q + 10.0 / 3.0 * pairs_q + 20.0 / 3.0 * pairs_kv)
 
 
-def oracle_run_sample(w, inputs, which: int, n: int) -> float:
+def oracle_run_sample(w, inputs, which: int, n: int, keep=None) -> float:
+    """Times the oracle on one sample; with `keep` (a list) also hands back the rows it computed."""
     from oracle import s2a_oracle as orc
 
     q, k, v, dO = inputs
     q_rows, kv_rows = oracle_sample_rows(w, which, n)
     t0 = time.perf_counter()
-    orc.fwd(q, k, v, w.G, rows=q_rows)
-    orc.bwd(q, k, v, dO, w.G, q_rows=q_rows, kv_rows=kv_rows)
-    return time.perf_counter() - t0
+    o_ref, lse_ref = orc.fwd(q, k, v, w.G, rows=q_rows)
+    dq_ref, dk_ref, dv_ref = orc.bwd(q, k, v, dO, w.G, q_rows=q_rows, kv_rows=kv_rows)
+    dt = time.perf_counter() - t0
+    if keep is not None:
+        keep.append((q_rows, kv_rows, o_ref, lse_ref, dq_ref, dk_ref, dv_ref))
+    return dt
 
 
-def time_oracle_steps(w, inputs, steps: int, warmup: int, n: int):
+def time_oracle_steps(w, inputs, steps: int, warmup: int, n: int, keep=None):
     from oracle import s2a_oracle as orc
 
     times = []
     for it in range(warmup + steps):
-        dt = oracle_run_sample(w, inputs, it, n)
+        dt = oracle_run_sample(w, inputs, it, n, keep if it >= warmup else None)
         if it >= warmup:
             times.append(dt)
     total = sum(times)
     return oracle_sample_flops(w, n) * steps / total / 1e12, total / steps, orc.num_threads()
+
+
+def parity_against_oracle(kept, gpu_out):
+    """Element-by-element comparison of the units the oracle just computed with what the GPU holds.
+
+    kept: [(q_rows, kv_rows, o, lse, dq, dk, dv)] from the oracle; gpu_out: the device tensors
+    (o, lse, dq, dk, dv) of the last step.  Returns max abs errors of o and lse, and for each gradient
+    the relative L2 error pooled over all compared rows and that of the worst single row (its norm
+    floored at 5 % of the rms row norm of its unit)."""
+    import numpy as np
+    import torch
+
+    o, lse, dq, dk, dv = gpu_out
+    res = {"o_max_abs": 0.0, "lse_max_abs": 0.0, "rows_q": 0, "rows_kv": 0}
+    pooled = {n: [0.0, 0.0] for n in ("dq", "dk", "dv")}
+    worst = {n: 0.0 for n in ("dq", "dk", "dv")}
+    for q_rows, kv_rows, o_ref, lse_ref, dq_ref, dk_ref, dv_ref in kept:
+        qi = torch.tensor(q_rows, device=o.device)
+        ki = torch.tensor(kv_rows, device=o.device)
+        got = {
+            "o": o[qi[:, 0], qi[:, 2], qi[:, 1]], "lse": lse[qi[:, 0], qi[:, 1], qi[:, 2]],
+            "dq": dq[qi[:, 0], qi[:, 2], qi[:, 1]], "dk": dk[ki[:, 0], ki[:, 2], ki[:, 1]],
+            "dv": dv[ki[:, 0], ki[:, 2], ki[:, 1]],
+        }
+        got = {n: x.double().cpu().numpy() for n, x in got.items()}
+        res["o_max_abs"] = max(res["o_max_abs"], float(np.abs(got["o"] - o_ref).max()))
+        res["lse_max_abs"] = max(res["lse_max_abs"], float(np.abs(got["lse"] - lse_ref).max()))
+        res["rows_q"] += len(q_rows)
+        res["rows_kv"] += len(kv_rows)
+        for n, ref in (("dq", dq_ref), ("dk", dk_ref), ("dv", dv_ref)):
+            diff2 = ((got[n] - ref) ** 2).sum(axis=-1)
+            ref2 = (ref ** 2).sum(axis=-1)
+            pooled[n][0] += float(diff2.sum())
+            pooled[n][1] += float(ref2.sum())
+            # a row's own norm, floored at 5 % of the rms row norm (the first row of a group has dq = 0 exactly)
+            floor2 = 0.0025 * float(ref2.mean())
+            worst[n] = max(worst[n], float(np.sqrt(diff2 / np.maximum(ref2, max(floor2, 1e-300))).max()))
+    for n in ("dq", "dk", "dv"):
+        res[f"{n}_rel_l2"] = (pooled[n][0] / max(pooled[n][1], 1e-300)) ** 0.5
+        res[f"{n}_rel_l2_worst_row"] = worst[n]
+    res["tolerance"] = {"o_max_abs": 2e-2, "grad_rel_l2": 1e-2}
+    res["ok"] = bool(res["o_max_abs"] <= 2e-2 and max(res["dq_rel_l2"], res["dk_rel_l2"], res["dv_rel_l2"]) <= 1e-2)
+    return res
 
 
 def run_reference(args):
@@ -242,8 +289,18 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    warmup = max(args.warmup, 3)   # the timing rules want at least three; the line reports what was run
+    if warmup != args.warmup and rank == 0:
+        print(f"bench.py: --warmup {args.warmup} raised to {warmup}", file=sys.stderr)
+    for _ in range(warmup):
         step_plain()
+    barrier()
+    # host side of a step: time spent in the entry points (argument checks, tensor maps, launches),
+    # nothing on the device waited for
+    t0 = time.perf_counter()
+    for _ in range(5):
+        step_plain()
+    host_us = (time.perf_counter() - t0) / 5 * 1e6
     barrier()
     rc, where = s2a.device_status()
     if rc != 0:
@@ -275,6 +332,7 @@ def run_ours(args):
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     total_ms = ev[0][0].elapsed_time(end)
+    step_ms = [ev[i][0].elapsed_time(ev[i + 1][0] if i + 1 < K else end) for i in range(K)]
     kernel_ms = {n: sum(ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(K)) for j, n in enumerate(names)}
     rc, where = s2a.device_status()
     if rc != 0:
@@ -326,26 +384,51 @@ def run_ours(args):
                       "algorithmic_tflops": alg_flops[n] / (ms * 1e-3) / 1e12 if ms > 0 else None,
                       "executed_tflops": exe_flops[n] / (ms * 1e-3) / 1e12 if ms > 0 else None}
     dom = max(names, key=lambda n: kernel_ms[n])
-    peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+    peak_sustained = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+    peak_burst = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
+    # Which measured peak this run is comparable with: the sustained one when the run itself was held
+    # back by the power cap (the reason was active, or the SM clock sat well below its maximum),
+    # the burst one when it ran at full clock throughout.
+    regime = "sustained"
+    if clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz"):
+        capped = "sw_power_cap" in clocks.get("reasons", []) or clocks["sm_mhz"] < 0.97 * clocks["sm_max_mhz"]
+        regime = "sustained" if capped else "burst"
+    peak = peak_sustained if regime == "sustained" else peak_burst
     achieved = kernels[dom]["algorithmic_tflops"]
     traffic = NCU_TRAFFIC_8K.get(dom)
     if traffic is not None:
         traffic = traffic * (B * N * (H + Hkv) * d) / NCU_TRAFFIC_8K_SIZE
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": traffic, "traffic_unit": "bytes per launch (ncu on 8k, scaled)",
-                "peak_source": f"{peak_src} bf16 sustained (burst {peaks.get('bf16_tflops')})",
-                "whole_step_frac": value / world / peak}
+                "peak_source": f"{peak_src} bf16 {regime} (chosen from this run's clock record)",
+                "frac_of_burst": achieved / peak_burst, "frac_of_sustained": achieved / peak_sustained,
+                "peaks": {"burst": peak_burst, "sustained": peak_sustained},
+                "whole_step_frac": value / world / peak,
+                "whole_step_frac_of_burst": value / world / peak_burst,
+                "whole_step_frac_of_sustained": value / world / peak_sustained}
 
     cpu_baseline = None
+    parity = None
     if world == 1 and not args.no_cpu_baseline:
-        tf, sec, cores = time_oracle_steps(w, host_in, steps=2, warmup=0, n=w.G)
+        kept = []
+        tf, sec, cores = time_oracle_steps(w, host_in, steps=2, warmup=0, n=w.G, keep=kept)
         cpu_baseline = {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle",
                         "sample": f"2 whole (batch, head, group) units of {w.name} (the shifted wrapped last group "
                                   f"of head {H - 1}, the first group of head 0), forward+backward, {sec:.1f} s each"}
+        # the same two units, every row of them, against the device path (the host-buffer entry point
+        # above used the device tensors, inputs included, as staging space: restore the inputs and run
+        # one more plain step)
+        for dst, src in zip((q, k, v, dO), host_in):
+            dst.copy_(src)
+        step_plain()
+        torch.cuda.synchronize()
+        parity = parity_against_oracle(kept, (o, lse, dq, dk, dv))
+        parity["sample"] = "every query row and key row of the two units of cpu_baseline"
 
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
-        "ms_per_step": total_ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": warmup,
+        "ms_per_step": total_ms_max / K, "ms_per_step_median": statistics.median(step_ms), "ms_per_step_best": min(step_ms),
+        "host_enqueue_us_per_step": host_us, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "B": B, "N": N, "G": G, "H": H, "Hkv": Hkv, "d": d,
                    "l2": "inputs (5 x %.0f MB) larger than L2" % (q.numel() * 2 / 1e6),
@@ -358,6 +441,7 @@ def run_ours(args):
         "roofline": roofline,
         "kernels": kernels,
         "cpu_baseline": cpu_baseline,
+        "parity": parity,
     }
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -376,7 +460,22 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return launch_ranks(args)
     return run_ours(args)
+
+
+def launch_ranks(args):
+    """`python bench.py --gpus N` without a launcher around it: start N ranks, one GPU each, under
+    torch.distributed.run on this node and let rank 0's JSON line through."""
+    import socket
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 if __name__ == "__main__":

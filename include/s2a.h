@@ -23,7 +23,12 @@
  *     lse          : fp32 [B, H, N]   natural-log sum-exp of the scaled scores, original token order
  *   - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).  Calls only enqueue
  *     work and return without synchronising.
- *   - Return value: S2A_OK (0) or a negative s2a_status.  On error nothing was enqueued.
+ *   - Return value: S2A_OK (0) or a negative s2a_status.  Arguments are checked before anything is
+ *     enqueued, so S2A_ERR_INVALID_ARG, S2A_ERR_UNSUPPORTED, S2A_ERR_TOO_LARGE and S2A_ERR_TIMEOUT mean
+ *     that nothing was enqueued.  S2A_ERR_CUDA means a CUDA call failed while enqueuing: an entry
+ *     point that makes several launches or copies (s2a_bwd and its variants, s2a_fwd_bwd_host) may by
+ *     then have enqueued the earlier ones, so the outputs are unspecified; `stream` still covers
+ *     everything that was enqueued (s2a_fwd_bwd_host joins its copy streams into it on every path).
  *   - Supported shapes: d in {64, 128}; N a multiple of G, N >= 128; G a multiple of 8 (so that every
  *     run of tokens of a group, shifted by G/2 or not, starts and ends on a multiple of 4 tokens);
  *     H even; H a multiple of Hkv; pointers 16-byte aligned; a device of compute capability 10.x.
@@ -31,13 +36,25 @@
  *     25,000): a group is then covered by tiles whose last one is partly masked, and the group that
  *     wraps around the end of the sequence by two such runs of tiles.  Anything else is rejected,
  *     never approximated.
- *   - Rows of a partly masked tile that belong to a neighbouring group are read (and masked), so a
- *     NaN or infinity in one token's k or v can reach the outputs of the adjacent group's tokens.
+ *   - Rows of a partly masked tile that belong to a neighbouring group are read and masked by
+ *     multiplying with zero weights, so inputs are assumed finite: where G or G/2 is not a multiple of
+ *     128, a NaN or infinity in one token's q, k, v or dO can reach o, dq, dk or dv of the adjacent
+ *     group's tokens.
  *   - Host threads: entry points may be called from several host threads (the one-time set-up of a
  *     device is serialised); s2a_fwd_bwd_host and s2a_bwd_noalloc keep per-device state (copy streams,
  *     built-in scratch), so calls of either on one device must not overlap.
- *   - Device-side waits are bounded.  If one ever expires the kernel records where, stops cleanly,
- *     and s2a_device_status() reports it; outputs of that launch are then undefined.
+ *   - Device-side waits are bounded (about a second of SM clock cycles, so heavy time-slicing of the
+ *     GPU can in principle trip one).  If a wait expires the kernel records where, in a status word on
+ *     the device and in a host-visible copy of it, and stops cleanly; the outputs of that launch are
+ *     undefined.  The status is STICKY: until s2a_device_status() has read and cleared it, every
+ *     kernel of this library that is already enqueued or gets launched on that device returns at once
+ *     without writing its outputs, and every entry point that would enqueue work returns
+ *     S2A_ERR_TIMEOUT instead (a host-side check of the copy; no synchronisation).  So a caller that
+ *     sees S2A_ERR_TIMEOUT calls s2a_device_status(), discards the results since the last clean
+ *     check, and goes on.
+ *   - The first call on a device sets the library up for it (kernel attributes, the address of the
+ *     status word, page-locking of a 4 KiB static status area); it allocates nothing, and should be
+ *     made outside any stream capture.
  */
 #ifndef S2A_H_
 #define S2A_H_
@@ -93,14 +110,13 @@ size_t s2a_bwd_workspace_bytes(int B, int N, int H, int Hkv, int d, int G);
  * on the same side of n_unshifted (n_unshifted a multiple of H/Hkv).  n_unshifted = H gives "pattern 1 only"; with G = N as well it is ordinary full
  * causal attention, which the fine-tuned model uses at inference.  `scale` multiplies the scores
  * (pass 1/sqrt(d) for the standard choice).  H may be odd here.
- * flags: S2A_FLAG_LEAK_FREE selects variant 2 of Appendix B ("individual groups for the shifted
- * tokens"): in a shifted head the group that wraps around the sequence end is cut in two at the
- * wrap, so the sequence's first tokens no longer attend its last tokens.
- * S2A_FLAG_SWAP_WRAPPED selects variant 3 ("swaps the shifted and the original front tokens"; its
- * figure is not in the paper's text, so this is a reading): in that same group the two parts change
- * places, i.e. the group is attended in original token order - the first tokens of the sequence, then
- * its last ones - so that no token attends a later one.  The two flags exclude each other; other bits
- * must be 0.
+ * flags: S2A_FLAG_LEAK_FREE selects variant 2 of Appendix B / Table 8: in a shifted head the group
+ * that wraps around the sequence end is cut in two at the wrap, so the sequence's first tokens no
+ * longer attend its last tokens.
+ * S2A_FLAG_SWAP_WRAPPED selects variant 3 of Appendix B / Table 8 (its figure is not in the paper's
+ * text, so this is a reading): in that same group the two parts change places, i.e. the group is
+ * attended in original token order - the first tokens of the sequence, then its last ones - so that
+ * no token attends a later one.  The two flags exclude each other; other bits must be 0.
  */
 #define S2A_FLAG_LEAK_FREE 1u
 #define S2A_FLAG_SWAP_WRAPPED 2u
@@ -176,9 +192,10 @@ int s2a_bwd_stage(const void* q, const void* k, const void* v, const void* o, co
 /*
  * Forward + backward from HOST buffers (pinned memory, or the copies are not asynchronous): q, k, v,
  * dO go to the caller's device buffers, s2a_fwd and s2a_bwd run there, and o, lse, dq, dk, dv come
- * back.  Heads are independent, so the work is cut into up to 8 chunks of whole KV heads and the
- * copy of one chunk, the kernels of the previous one and the copy back of the one before that
- * overlap (two copy streams owned by the library, created by the first call on a device, ordered
+ * back.  Heads are independent, so the work is cut into up to 16 chunks of whole KV heads - one KV head
+ * at either end, growing towards the middle - and the copy of one chunk, the kernels of the previous
+ * one and the copy back of the one before that overlap (two copy streams owned by the library,
+ * created by the first call on a device, ordered
  * against `stream` by events).  Everything is ordered after the work already in `stream` and
  * `stream` is complete only when the last result has landed: the caller synchronises `stream`
  * before reading the host outputs.  Results are bit-identical to s2a_fwd + s2a_bwd.
@@ -192,6 +209,16 @@ int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const vo
                      void* d_dq, void* d_dk, void* d_dv,
                      int B, int N, int H, int Hkv, int d, int G,
                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Diagnostic (the paper has no counterpart): enqueues one tiny kernel on `stream` in which a single
+ * warp waits, with the library's own bounded wait and a limit of `limit_cycles` SM clock cycles
+ * (1 .. 2,000,000,000; a million is well under a millisecond), on a barrier that nothing ever arrives
+ * on.  The wait runs out, the kernel reports it exactly as a production kernel would (wait code 901)
+ * and returns; nothing hangs and nothing faults.  It lets a caller, or a test, see the whole
+ * time-out path: the sticky status, S2A_ERR_TIMEOUT from the entry points, s2a_device_status().
+ */
+int s2a_selftest_wait_expiry(long long limit_cycles, void* stream);
 
 /*
  * Reads (and clears) the device-side status word of the current device.  Synchronises the device.

@@ -61,10 +61,10 @@ def _swap_halves_of_wrapped_group(x, B, n_groups, H):
 
 def s2_attn(q, k, v, G, scale=None, leak_free=False, swap_wrapped=False):
     """q [B,N,H,d], k/v [B,N,Hkv,d] (fp64) -> o [B,N,H,d], lse [B,H,N].
-    leak_free: variant 2 of Appendix B ("a small modification on the attention mask"): in the shifted
+    leak_free: variant 2 of Appendix B (Table 8; done there by changing the attention mask): in the shifted
     heads the last group, which holds the sequence's last G/2 tokens followed by its first G/2 tokens,
     is treated as two groups, so the front tokens do not attend the tail tokens.
-    swap_wrapped: variant 3 of Appendix B ("swaps the shifted and the original front tokens"): in that same
+    swap_wrapped: variant 3 of Appendix B (Table 8; front and shifted tokens exchanged): in that same
     group the two halves change places before the attention and change back after it, so the group is
     attended in original token order (front tokens first)."""
     B, N, H, d = q.shape

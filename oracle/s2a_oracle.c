@@ -100,9 +100,9 @@ static int head_shift(const s2a_dims* D, int h) { return h < D->n_unshifted ? 0 
  * Variants 2 and 3 of Appendix B concern the one group of a shifted head that wraps around the
  * sequence end: it holds the last tokens of the sequence ("tail") followed by the first ones
  * ("front"), so that in Algorithm 1 the front tokens attend the tail tokens.
- *   variant 2 ("uses individual groups for the shifted tokens"): the group is cut in two at the wrap;
+ *   variant 2 (Appendix B, Table 8; separate groups for the shifted tokens): the group is cut in two at the wrap;
  *             front tokens attend front tokens only, tail tokens attend tail tokens only.
- *   variant 3 ("swaps the shifted and the original front tokens"): the two parts change places, so
+ *   variant 3 (Appendix B, Table 8; the front and the shifted tokens exchanged): the two parts change places, so
  *             the group is in original token order: front tokens come first (and attend only
  *             themselves), tail tokens follow and attend all front tokens and the tail tokens before
  *             them.

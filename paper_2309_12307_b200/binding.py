@@ -25,7 +25,7 @@ S2A_ERR_TOO_LARGE = -5
 EXPORTS = [
     "s2a_fwd", "s2a_bwd", "s2a_bwd_workspace_bytes", "s2a_fwd_ex", "s2a_bwd_ex", "s2a_bwd_stage", "s2a_fwd_bwd_host",
     "s2a_bwd_noalloc", "s2a_bwd_noalloc_max_rows", "s2a_fwd_packed", "s2a_bwd_packed",
-    "s2a_device_status", "s2a_status_string", "s2a_last_cuda_error", "s2a_version",
+    "s2a_selftest_wait_expiry", "s2a_device_status", "s2a_status_string", "s2a_last_cuda_error", "s2a_version",
 ]
 
 _lib = None
@@ -68,6 +68,8 @@ def load() -> ctypes.CDLL:
     lib.s2a_bwd_workspace_bytes.restype = Z
     lib.s2a_fwd_bwd_host.argtypes = [P] * 18 + [I] * 6 + [P, Z, P]
     lib.s2a_fwd_bwd_host.restype = I
+    lib.s2a_selftest_wait_expiry.argtypes = [ctypes.c_longlong, P]
+    lib.s2a_selftest_wait_expiry.restype = I
     lib.s2a_device_status.argtypes = [ctypes.POINTER(I)]
     lib.s2a_device_status.restype = I
     lib.s2a_status_string.argtypes = [I]
@@ -101,14 +103,54 @@ def _check(rc: int, what: str) -> None:
         raise S2AError(rc, what)
 
 
-def _dims(q: torch.Tensor, k: torch.Tensor):
+def _require(t, dtype, name: str, shape=None, device=None, cuda: bool = True):
+    """One tensor the library will read or write through its raw pointer: it must be what the C side
+    takes it for, or the kernels would reinterpret foreign memory."""
+    if not isinstance(t, torch.Tensor):
+        raise ValueError(f"{name} must be a torch.Tensor")
+    if t.is_cuda != cuda:
+        raise ValueError(f"{name} must be a {'CUDA' if cuda else 'CPU (pinned)'} tensor")
+    if t.dtype != dtype:
+        raise ValueError(f"{name} must have dtype {dtype}, not {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} must have shape {tuple(shape)}, not {tuple(t.shape)}")
+    if device is not None and t.device != device:
+        raise ValueError(f"{name} must be on {device}, not {t.device}")
+
+
+def _dims(q, k, v, cuda: bool = True):
+    """Checks q [B,N,H,d] and k, v [B,N,Hkv,d] (bf16, contiguous, one device) and returns the sizes."""
+    _require(q, torch.bfloat16, "q", cuda=cuda)
+    if q.dim() != 4:
+        raise ValueError(f"q must be [B, N, H, d], not {tuple(q.shape)}")
     B, N, H, d = q.shape
-    return B, N, H, k.shape[2], d
+    _require(k, torch.bfloat16, "k", device=q.device, cuda=cuda)
+    if k.dim() != 4 or k.shape[0] != B or k.shape[1] != N or k.shape[3] != d:
+        raise ValueError(f"k must be [B, N, Hkv, d] = [{B}, {N}, Hkv, {d}], not {tuple(k.shape)}")
+    Hkv = k.shape[2]
+    _require(v, torch.bfloat16, "v", shape=k.shape, device=q.device, cuda=cuda)
+    return B, N, H, Hkv, d
 
 
-def _require(t: torch.Tensor, dtype, name: str):
-    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
-        raise ValueError(f"{name} must be a contiguous CUDA tensor of dtype {dtype}")
+def _check_fwd_out(q, o, lse):
+    B, N, H, d = q.shape
+    _require(o, torch.bfloat16, "o", shape=q.shape, device=q.device)
+    _require(lse, torch.float32, "lse", shape=(B, H, N), device=q.device)
+
+
+def _check_bwd(q, k, o, lse, dO, dq, dk, dv):
+    _check_fwd_out(q, o, lse)
+    _require(dO, torch.bfloat16, "dO", shape=q.shape, device=q.device)
+    _require(dq, torch.bfloat16, "dq", shape=q.shape, device=q.device)
+    _require(dk, torch.bfloat16, "dk", shape=k.shape, device=q.device)
+    _require(dv, torch.bfloat16, "dv", shape=k.shape, device=q.device)
+
+
+def _check_workspace(ws, device):
+    """The workspace's size is checked by the library (S2A_ERR_INVALID_ARG); here only what it is."""
+    _require(ws, torch.uint8, "workspace", device=device)
 
 
 def bwd_workspace_bytes(B, N, H, Hkv, d, G) -> int:
@@ -117,15 +159,12 @@ def bwd_workspace_bytes(B, N, H, Hkv, d, G) -> int:
 
 def s2a_fwd(q, k, v, G, o=None, lse=None, stream=None):
     """o [B,N,H,d] bf16 and lse [B,H,N] fp32 of S2-Attn (second half of the heads shifted by G/2)."""
-    B, N, H, Hkv, d = _dims(q, k)
-    for t, n in ((q, "q"), (k, "k"), (v, "v")):
-        _require(t, torch.bfloat16, n)
+    B, N, H, Hkv, d = _dims(q, k, v)
     if o is None:
         o = torch.empty_like(q)
     if lse is None:
         lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device)
-    _require(o, torch.bfloat16, "o")
-    _require(lse, torch.float32, "lse")
+    _check_fwd_out(q, o, lse)
     rc = load().s2a_fwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), B, N, H, Hkv, d, G,
                         _stream_ptr(stream))
     _check(rc, "s2a_fwd")
@@ -134,16 +173,15 @@ def s2a_fwd(q, k, v, G, o=None, lse=None, stream=None):
 
 def s2a_bwd(q, k, v, o, lse, dO, G, dq=None, dk=None, dv=None, workspace=None, stream=None):
     """dq, dk, dv (bf16) of sum(o * dO)."""
-    B, N, H, Hkv, d = _dims(q, k)
-    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (dO, "dO")):
-        _require(t, torch.bfloat16, n)
-    _require(lse, torch.float32, "lse")
+    B, N, H, Hkv, d = _dims(q, k, v)
     dq = torch.empty_like(q) if dq is None else dq
     dk = torch.empty_like(k) if dk is None else dk
     dv = torch.empty_like(v) if dv is None else dv
+    _check_bwd(q, k, o, lse, dO, dq, dk, dv)
     need = bwd_workspace_bytes(B, N, H, Hkv, d, G)
     if workspace is None:
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    _check_workspace(workspace, q.device)
     rc = load().s2a_bwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), dO.data_ptr(),
                         dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, N, H, Hkv, d, G, workspace.data_ptr(),
                         workspace.numel() * workspace.element_size(), _stream_ptr(stream))
@@ -162,7 +200,8 @@ def s2a_bwd_noalloc(q, k, v, o, lse, dO, G, dq, dk, dv, stream=None):
     tensor.  B*H*N must not exceed bwd_noalloc_max_rows().  Calls that may overlap on the GPU
     share the array and must be serialised (see include/s2a.h).
     """
-    B, N, H, Hkv, d = _dims(q, k)
+    B, N, H, Hkv, d = _dims(q, k, v)
+    _check_bwd(q, k, o, lse, dO, dq, dk, dv)
     rc = load().s2a_bwd_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(),
                                 dO.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, N, H, Hkv, d, G,
                                 _stream_ptr(stream))
@@ -170,13 +209,21 @@ def s2a_bwd_noalloc(q, k, v, o, lse, dO, G, dq, dk, dv, stream=None):
     return dq, dk, dv
 
 
+def _packed_dims(qkv):
+    _require(qkv, torch.bfloat16, "qkv")
+    if qkv.dim() != 5 or qkv.shape[2] != 3:
+        raise ValueError(f"qkv must be [B, N, 3, H, d], not {tuple(qkv.shape)}")
+    B, N, _, H, d = qkv.shape
+    return B, N, H, d
+
+
 def s2a_fwd_packed(qkv, G, o=None, lse=None, stream=None):
     """Forward on a packed qkv tensor [B, N, 3, H, d] (the calling convention of Algorithm 1)."""
-    B, N, three, H, d = qkv.shape
-    assert three == 3
-    _require(qkv, torch.bfloat16, "qkv")
+    B, N, H, d = _packed_dims(qkv)
     o = torch.empty((B, N, H, d), dtype=torch.bfloat16, device=qkv.device) if o is None else o
     lse = torch.empty((B, H, N), dtype=torch.float32, device=qkv.device) if lse is None else lse
+    _require(o, torch.bfloat16, "o", shape=(B, N, H, d), device=qkv.device)
+    _require(lse, torch.float32, "lse", shape=(B, H, N), device=qkv.device)
     rc = load().s2a_fwd_packed(qkv.data_ptr(), o.data_ptr(), lse.data_ptr(), B, N, H, d, G, _stream_ptr(stream))
     _check(rc, "s2a_fwd_packed")
     return o, lse
@@ -184,12 +231,16 @@ def s2a_fwd_packed(qkv, G, o=None, lse=None, stream=None):
 
 def s2a_bwd_packed(qkv, o, lse, dO, G, dqkv=None, workspace=None, stream=None):
     """Backward on a packed qkv tensor; returns dqkv [B, N, 3, H, d]."""
-    B, N, three, H, d = qkv.shape
-    assert three == 3
+    B, N, H, d = _packed_dims(qkv)
     dqkv = torch.empty_like(qkv) if dqkv is None else dqkv
+    _require(dqkv, torch.bfloat16, "dqkv", shape=qkv.shape, device=qkv.device)
+    _require(o, torch.bfloat16, "o", shape=(B, N, H, d), device=qkv.device)
+    _require(dO, torch.bfloat16, "dO", shape=(B, N, H, d), device=qkv.device)
+    _require(lse, torch.float32, "lse", shape=(B, H, N), device=qkv.device)
     need = bwd_workspace_bytes(B, N, H, H, d, G)
     if workspace is None:
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=qkv.device)
+    _check_workspace(workspace, qkv.device)
     rc = load().s2a_bwd_packed(qkv.data_ptr(), o.data_ptr(), lse.data_ptr(), dO.data_ptr(), dqkv.data_ptr(), B, N, H, d, G,
                                workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     _check(rc, "s2a_bwd_packed")
@@ -198,7 +249,9 @@ def s2a_bwd_packed(qkv, o, lse, dO, G, dqkv=None, workspace=None, stream=None):
 
 def s2a_bwd_stage(q, k, v, o, lse, dO, G, dq, dk, dv, workspace, stage, stream=None):
     """Enqueue one kernel of the backward: 0 = D preprocess, 1 = dk/dv, 2 = dq (profiling aid)."""
-    B, N, H, Hkv, d = _dims(q, k)
+    B, N, H, Hkv, d = _dims(q, k, v)
+    _check_bwd(q, k, o, lse, dO, dq, dk, dv)
+    _check_workspace(workspace, q.device)
     rc = load().s2a_bwd_stage(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), dO.data_ptr(),
                               dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, N, H, Hkv, d, G, workspace.data_ptr(),
                               workspace.numel() * workspace.element_size(), int(stage), _stream_ptr(stream))
@@ -218,12 +271,13 @@ def s2a_fwd_ex(q, k, v, G, scale=None, n_unshifted=None, shift=None, leak_free=F
     """Generalised forward: heads [0, n_unshifted) unshifted, the rest rolled by -shift tokens;
     leak_free=True cuts the wrapped group of the shifted heads at the wrap (Appendix B, variant 2);
     swap_wrapped=True makes its two parts change places (variant 3)."""
-    B, N, H, Hkv, d = _dims(q, k)
+    B, N, H, Hkv, d = _dims(q, k, v)
     scale = 1.0 / math.sqrt(d) if scale is None else scale
     n_unshifted = H // 2 if n_unshifted is None else n_unshifted
     shift = G // 2 if shift is None else shift
     o = torch.empty_like(q) if o is None else o
     lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if lse is None else lse
+    _check_fwd_out(q, o, lse)
     rc = load().s2a_fwd_ex(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), B, N, H, Hkv, d, G,
                            scale, n_unshifted, shift, _flags(leak_free, swap_wrapped), _stream_ptr(stream))
     _check(rc, "s2a_fwd_ex")
@@ -232,16 +286,18 @@ def s2a_fwd_ex(q, k, v, G, scale=None, n_unshifted=None, shift=None, leak_free=F
 
 def s2a_bwd_ex(q, k, v, o, lse, dO, G, scale=None, n_unshifted=None, shift=None, leak_free=False, workspace=None,
                stream=None, dq=None, dk=None, dv=None, swap_wrapped=False):
-    B, N, H, Hkv, d = _dims(q, k)
+    B, N, H, Hkv, d = _dims(q, k, v)
     scale = 1.0 / math.sqrt(d) if scale is None else scale
     n_unshifted = H // 2 if n_unshifted is None else n_unshifted
     shift = G // 2 if shift is None else shift
     dq = torch.empty_like(q) if dq is None else dq
     dk = torch.empty_like(k) if dk is None else dk
     dv = torch.empty_like(v) if dv is None else dv
+    _check_bwd(q, k, o, lse, dO, dq, dk, dv)
     need = bwd_workspace_bytes(B, N, H, Hkv, d, G)
     if workspace is None:
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    _check_workspace(workspace, q.device)
     rc = load().s2a_bwd_ex(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), dO.data_ptr(),
                            dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, N, H, Hkv, d, G, scale, n_unshifted, shift,
                            _flags(leak_free, swap_wrapped), workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
@@ -258,11 +314,26 @@ def s2a_fwd_bwd_host(host_in, host_out, dev, G, workspace, stream=None):
     """
     hq, hk, hv, hdo = host_in
     ho, hlse, hdq, hdk, hdv = host_out
-    B, N, H, Hkv, d = _dims(hq, hk)
+    B, N, H, Hkv, d = _dims(hq, hk, hv, cuda=False)
+    bf, f32 = torch.bfloat16, torch.float32
+    for t, name, dt, shp in ((hdo, "host dO", bf, hq.shape), (ho, "host o", bf, hq.shape), (hlse, "host lse", f32, (B, H, N)),
+                             (hdq, "host dq", bf, hq.shape), (hdk, "host dk", bf, hk.shape), (hdv, "host dv", bf, hk.shape)):
+        _require(t, dt, name, shape=shp, cuda=False)
+    if len(dev) != 9:
+        raise ValueError("dev must hold the nine device buffers (q, k, v, dO, o, lse, dq, dk, dv)")
+    shapes = (hq.shape, hk.shape, hk.shape, hq.shape, hq.shape, (B, H, N), hq.shape, hk.shape, hk.shape)
+    for t, shp, name in zip(dev, shapes, ("q", "k", "v", "dO", "o", "lse", "dq", "dk", "dv")):
+        _require(t, f32 if name == "lse" else bf, f"device {name}", shape=shp, device=dev[0].device)
+    _check_workspace(workspace, dev[0].device)
     ptrs = [t.data_ptr() for t in (hq, hk, hv, hdo, ho, hlse, hdq, hdk, hdv)] + [t.data_ptr() for t in dev]
     rc = load().s2a_fwd_bwd_host(*ptrs, B, N, H, Hkv, d, G, workspace.data_ptr(),
                                  workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     _check(rc, "s2a_fwd_bwd_host")
+
+
+def selftest_wait_expiry(limit_cycles: int = 1_000_000, stream=None) -> None:
+    """Enqueue the diagnostic kernel whose bounded wait runs out after `limit_cycles` SM cycles."""
+    _check(load().s2a_selftest_wait_expiry(int(limit_cycles), _stream_ptr(stream)), "s2a_selftest_wait_expiry")
 
 
 def device_status():

@@ -10,6 +10,7 @@
 
 #include "../../include/s2a.h"
 #include "s2a_params.h"
+#include "sm100_ptx.cuh"
 
 namespace s2a {
 namespace {
@@ -18,20 +19,32 @@ namespace {
 // that loads this library).
 __device__ int g_status_word;
 
+// Host-visible mirrors of the status words, one per device (64 bytes apart): page-locked and mapped
+// into the device address space, so that a kernel can store the code of an expired wait where the
+// next entry point sees it without synchronising.  This is ordinary static memory, pinned in place
+// once per process; nothing is allocated.
+constexpr int kMirrorStride = 16;  // ints
+constexpr int kMaxDevicesMirror = 64;
+alignas(4096) int g_host_status[kMaxDevicesMirror * kMirrorStride];
+bool g_host_status_registered = false;
+
 thread_local int tl_last_cuda_error = 0;
 
 constexpr int kMaxDevices = 64;
-constexpr int kMaxHostChunks = 8;
+constexpr int kMaxHostChunks = 16;
 struct DeviceState {
     bool ready = false;
-    int* status_ptr = nullptr;
+    int* status_ptr = nullptr;        // device address of g_status_word
+    volatile int* host_word = nullptr;  // this device's mirror, host address
+    int* host_word_dev = nullptr;     // the same word as the device sees it
     // s2a_fwd_bwd_host only: copy streams and the events that order them against the caller's stream
     bool host_path_ready = false;
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
-    cudaEvent_t ev_start = nullptr, ev_done = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_done = nullptr, ev_in_done = nullptr;
     cudaEvent_t ev_in[kMaxHostChunks] = {}, ev_compute[kMaxHostChunks] = {};
 };
 DeviceState g_dev[kMaxDevices];
+static_assert(kMaxDevices == kMaxDevicesMirror, "one mirror word per device");
 std::mutex g_dev_mutex;  // guards the one-time set-up of a DeviceState (calls may come from several host threads)
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -70,6 +83,14 @@ int prepare_device(DeviceState** out) {
         e = configure_bwd();
         if (e != cudaSuccess) return cuda_fail(e);
         e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ds.status_ptr), g_status_word);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (!g_host_status_registered) {
+            e = cudaHostRegister(g_host_status, sizeof g_host_status, cudaHostRegisterPortable | cudaHostRegisterMapped);
+            if (e != cudaSuccess) return cuda_fail(e);
+            g_host_status_registered = true;
+        }
+        ds.host_word = &g_host_status[dev * kMirrorStride];
+        e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&ds.host_word_dev), const_cast<int*>(ds.host_word), 0);
         if (e != cudaSuccess) return cuda_fail(e);
         ds.ready = true;
     }
@@ -154,6 +175,24 @@ Geometry make_geometry(int B, int N, int H, int Hkv, int G, int n_unshifted, int
 
 constexpr float kLog2eHost = 1.4426950408889634f;
 
+// Diagnostic kernel behind s2a_selftest_wait_expiry: one warp waits, with the library's own bounded
+// wait and the given limit, on a barrier nothing ever arrives on.  The wait runs out, the expiry is
+// reported exactly as a production kernel reports one, and the kernel returns.
+constexpr int kWaitSelfTest = 900;
+__global__ void __launch_bounds__(32) s2a_wait_selftest_kernel(int* status, int* host_status, long long limit) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (*reinterpret_cast<volatile int*>(status) != 0) return;  // like every kernel here: a set status word means "do nothing"
+    const WaitCtx ctx{&abort_flag, status, host_status};
+    mbar_wait_limit(&bar, 0, ctx, kWaitSelfTest + 1, limit);
+}
+
 }  // namespace
 }  // namespace s2a
 
@@ -162,7 +201,7 @@ using namespace s2a;
 #pragma GCC visibility push(default)
 extern "C" {
 
-int s2a_version(void) { return 100; }
+int s2a_version(void) { return 200; }
 
 int s2a_last_cuda_error(void) { return tl_last_cuda_error; }
 
@@ -194,6 +233,7 @@ int fwd_impl(const void* q, const void* k, const void* v, void* o, float* lse, i
     DeviceState* ds = nullptr;
     rc = prepare_device(&ds);
     if (rc != S2A_OK) return rc;
+    if (*ds->host_word != 0) return S2A_ERR_TIMEOUT;  // an earlier launch gave up: see s2a_device_status()
 
     FwdParams p;
     memset(&p, 0, sizeof p);
@@ -203,6 +243,7 @@ int fwd_impl(const void* q, const void* k, const void* v, void* o, float* lse, i
     p.o = static_cast<__nv_bfloat16*>(o);
     p.lse = lse;
     p.status = ds->status_ptr;
+    p.host_status = ds->host_word_dev;
     p.geo = make_geometry(B, N, H, Hkv, G, n_unshifted, shift, flags);
     p.scale_log2 = scale * kLog2eHost;
     cudaError_t e = launch_fwd(p, d, static_cast<cudaStream_t>(stream));
@@ -257,6 +298,7 @@ int bwd_impl(const void* q, const void* k, const void* v, const void* o, const f
     DeviceState* ds = nullptr;
     rc = prepare_device(&ds);
     if (rc != S2A_OK) return rc;
+    if (*ds->host_word != 0) return S2A_ERR_TIMEOUT;  // an earlier launch gave up: see s2a_device_status()
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (!flags_ok(flags)) return S2A_ERR_INVALID_ARG;
     const Geometry geo = make_geometry(B, N, H, Hkv, G, n_unshifted, shift, flags);
@@ -270,7 +312,7 @@ int bwd_impl(const void* q, const void* k, const void* v, const void* o, const f
     if ((rc = make_tmap(&pq.tm_v, v, d, Hkv, N, B, kTile, ts.kv)) != S2A_OK) return rc;
     pq.dq_tok_stride = ts.dq ? ts.dq : static_cast<long long>(H) * d;
     pq.lse = lse, pq.Dsum = Dsum, pq.dq = static_cast<__nv_bfloat16*>(dq);
-    pq.status = ds->status_ptr, pq.geo = geo, pq.scale = scale, pq.scale_log2 = scale * kLog2eHost;
+    pq.status = ds->status_ptr, pq.host_status = ds->host_word_dev, pq.geo = geo, pq.scale = scale, pq.scale_log2 = scale * kLog2eHost;
 
     BwdDkDvParams pk;
     memset(&pk, 0, sizeof pk);
@@ -281,7 +323,7 @@ int bwd_impl(const void* q, const void* k, const void* v, const void* o, const f
     pk.dkv_tok_stride = ts.dkv ? ts.dkv : static_cast<long long>(Hkv) * d;
     pk.lse = lse, pk.Dsum = Dsum;
     pk.dk = static_cast<__nv_bfloat16*>(dk), pk.dv = static_cast<__nv_bfloat16*>(dv);
-    pk.status = ds->status_ptr, pk.geo = geo, pk.scale = scale, pk.scale_log2 = scale * kLog2eHost;
+    pk.status = ds->status_ptr, pk.host_status = ds->host_word_dev, pk.geo = geo, pk.scale = scale, pk.scale_log2 = scale * kLog2eHost;
 
     PreParams pp;
     pp.o = static_cast<const __nv_bfloat16*>(o), pp.dO = static_cast<const __nv_bfloat16*>(dO), pp.Dsum = Dsum;
@@ -360,6 +402,7 @@ int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const vo
         if ((e = cudaStreamCreateWithFlags(&ds->copy_out, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
         if ((e = cudaEventCreateWithFlags(&ds->ev_start, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
         if ((e = cudaEventCreateWithFlags(&ds->ev_done, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventCreateWithFlags(&ds->ev_in_done, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
         for (int c = 0; c < kMaxHostChunks; ++c) {
             if ((e = cudaEventCreateWithFlags(&ds->ev_in[c], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaEventCreateWithFlags(&ds->ev_compute[c], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
@@ -369,60 +412,99 @@ int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const vo
     lock.unlock();
     // Heads are independent, so the job is cut into chunks of whole KV heads (with their query heads):
     // while chunk c is computed, chunk c+1 travels to the device and the results of chunk c-1 travel
-    // back.  A chunk sits densely ([B, N, heads of the chunk, d]) in its share of the caller's buffers.
-    int chunks = 1;
-    for (int c = kMaxHostChunks; c > 1; c >>= 1) {
-        if (Hkv % c == 0) {
-            chunks = c;
-            break;
-        }
-    }
+    // back.  Only the first chunk's upload and the last chunk's download cannot be hidden, so the
+    // chunks at both ends are small (one KV head) and grow towards the middle, where wide rows keep
+    // the strided copies efficient: 1,1,2,4,8,8,4,2,1,1 KV heads for Hkv = 32.  Chunk c holds the KV
+    // heads [kv0[c], kv0[c] + kvn[c]) and sits densely ([B, N, heads of the chunk, d]) at the matching
+    // offset of the caller's device buffers.
     const int rep = H / Hkv;
-    const int kvc = Hkv / chunks, hc = kvc * rep;  // KV heads and query heads per chunk
+    int kv0[kMaxHostChunks], kvn[kMaxHostChunks];
+    int chunks = 0;
+    {
+        int left[kMaxHostChunks / 2], right[kMaxHostChunks / 2], nl = 0, nr = 0;
+        int remaining = Hkv, size = 1, uses = 0;
+        const int cap = Hkv >= 8 ? Hkv / 4 : 1;
+        while (remaining > 0) {
+            const int a = size < remaining ? size : remaining;
+            if (nl <= nr) left[nl++] = a; else right[nr++] = a;
+            remaining -= a;
+            if (++uses == (size == 1 ? 4 : 2)) {   // 1,1 at each end, then every size once per end
+                uses = 0;
+                if (size * 2 <= cap) size *= 2;
+            }
+            if (nl + nr == kMaxHostChunks - 1 && remaining > 0) {   // out of slots: the rest in one chunk
+                if (nl <= nr) left[nl++] = remaining; else right[nr++] = remaining;
+                remaining = 0;
+            }
+        }
+        int at_kv = 0;
+        for (int x = 0; x < nl; ++x) kv0[chunks] = at_kv, kvn[chunks] = left[x], at_kv += left[x], ++chunks;
+        for (int x = nr - 1; x >= 0; --x) kv0[chunks] = at_kv, kvn[chunks] = right[x], at_kv += right[x], ++chunks;
+    }
     const size_t rows = static_cast<size_t>(B) * N;
-    const size_t wq = static_cast<size_t>(hc) * d * 2, wk = static_cast<size_t>(kvc) * d * 2;  // bytes per token
+    const size_t hb = static_cast<size_t>(d) * 2;                                              // bytes of one head of one token
     const size_t pq = static_cast<size_t>(H) * d * 2, pk = static_cast<size_t>(Hkv) * d * 2;   // host pitches
-    const size_t wl = static_cast<size_t>(hc) * N * sizeof(float), pl = static_cast<size_t>(H) * N * sizeof(float);
+    const size_t pl = static_cast<size_t>(H) * N * sizeof(float);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     auto at = [](const void* base, size_t bytes) { return const_cast<char*>(static_cast<const char*>(base)) + bytes; };
 
     if ((e = cudaEventRecord(ds->ev_start, st)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaStreamWaitEvent(ds->copy_in, ds->ev_start, 0)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaStreamWaitEvent(ds->copy_out, ds->ev_start, 0)) != cudaSuccess) return cuda_fail(e);
-    for (int c = 0; c < chunks; ++c) {
-        const size_t oq = c * rows * wq, ok_ = c * rows * wk, ol = static_cast<size_t>(c) * B * wl;
-        void *cq = at(d_q, oq), *ck = at(d_k, ok_), *cv = at(d_v, ok_), *cdo = at(d_dO, oq), *co = at(d_o, oq);
-        void *cdq = at(d_dq, oq), *cdk = at(d_dk, ok_), *cdv = at(d_dv, ok_);
-        float* cl = reinterpret_cast<float*>(at(d_lse, ol));
-        // host -> device: the chunk's heads of every token
-        if ((e = cudaMemcpy2DAsync(cq, wq, at(h_q, c * wq), pq, wq, rows, cudaMemcpyHostToDevice, ds->copy_in)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpy2DAsync(ck, wk, at(h_k, c * wk), pk, wk, rows, cudaMemcpyHostToDevice, ds->copy_in)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpy2DAsync(cv, wk, at(h_v, c * wk), pk, wk, rows, cudaMemcpyHostToDevice, ds->copy_in)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpy2DAsync(cdo, wq, at(h_dO, c * wq), pq, wq, rows, cudaMemcpyHostToDevice, ds->copy_in)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaEventRecord(ds->ev_in[c], ds->copy_in)) != cudaSuccess) return cuda_fail(e);
-        // compute on the caller's stream; the second half of ALL heads is shifted
-        if ((e = cudaStreamWaitEvent(st, ds->ev_in[c], 0)) != cudaSuccess) return cuda_fail(e);
-        int n_unshifted = H / 2 - c * hc;
-        n_unshifted = n_unshifted < 0 ? 0 : (n_unshifted > hc ? hc : n_unshifted);
-        const float scale = 1.0f / sqrtf(static_cast<float>(d));
-        rc = fwd_impl(cq, ck, cv, co, cl, B, N, hc, kvc, d, G, scale, n_unshifted, G / 2, 0u, stream, TokStrides());
-        if (rc != S2A_OK) return rc;
-        rc = bwd_impl(cq, ck, cv, co, cl, cdo, cdq, cdk, cdv, B, N, hc, kvc, d, G, scale, n_unshifted, G / 2, workspace,
-                      workspace_bytes, stream, kStageAll);
-        if (rc != S2A_OK) return rc;
-        if ((e = cudaEventRecord(ds->ev_compute[c], st)) != cudaSuccess) return cuda_fail(e);
-        // device -> host
-        if ((e = cudaStreamWaitEvent(ds->copy_out, ds->ev_compute[c], 0)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpy2DAsync(at(h_o, c * wq), pq, co, wq, wq, rows, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpy2DAsync(at(h_lse, c * wl), pl, cl, wl, wl, B, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpy2DAsync(at(h_dq, c * wq), pq, cdq, wq, wq, rows, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpy2DAsync(at(h_dk, c * wk), pk, cdk, wk, wk, rows, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpy2DAsync(at(h_dv, c * wk), pk, cdv, wk, wk, rows, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
+    // From here on work may sit in the two copy streams: whatever happens, `stream` is made to wait
+    // for both before this function returns, so that the caller's synchronisation covers it all.
+    auto join = [&]() -> cudaError_t {
+        cudaError_t e1 = cudaEventRecord(ds->ev_done, ds->copy_out);
+        if (e1 == cudaSuccess) e1 = cudaStreamWaitEvent(st, ds->ev_done, 0);
+        cudaError_t e2 = cudaEventRecord(ds->ev_in_done, ds->copy_in);
+        if (e2 == cudaSuccess) e2 = cudaStreamWaitEvent(st, ds->ev_in_done, 0);
+        return e1 != cudaSuccess ? e1 : e2;
+    };
+    auto enqueue_all = [&]() -> int {
+        if ((e = cudaStreamWaitEvent(ds->copy_in, ds->ev_start, 0)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamWaitEvent(ds->copy_out, ds->ev_start, 0)) != cudaSuccess) return cuda_fail(e);
+        for (int c = 0; c < chunks; ++c) {
+            const int kvc = kvn[c], hc = kvc * rep, h0 = kv0[c] * rep;   // KV heads, query heads, first query head of the chunk
+            const size_t wq = hc * hb, wk = kvc * hb;                    // bytes per token of the chunk
+            const size_t wl = static_cast<size_t>(hc) * N * sizeof(float);
+            const size_t oq = rows * h0 * hb, ok_ = rows * kv0[c] * hb, ol = static_cast<size_t>(B) * h0 * N * sizeof(float);
+            void *cq = at(d_q, oq), *ck = at(d_k, ok_), *cv = at(d_v, ok_), *cdo = at(d_dO, oq), *co = at(d_o, oq);
+            void *cdq = at(d_dq, oq), *cdk = at(d_dk, ok_), *cdv = at(d_dv, ok_);
+            float* cl = reinterpret_cast<float*>(at(d_lse, ol));
+            // host -> device: the chunk's heads of every token
+            if ((e = cudaMemcpy2DAsync(cq, wq, at(h_q, h0 * hb), pq, wq, rows, cudaMemcpyHostToDevice, ds->copy_in)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaMemcpy2DAsync(ck, wk, at(h_k, kv0[c] * hb), pk, wk, rows, cudaMemcpyHostToDevice, ds->copy_in)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaMemcpy2DAsync(cv, wk, at(h_v, kv0[c] * hb), pk, wk, rows, cudaMemcpyHostToDevice, ds->copy_in)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaMemcpy2DAsync(cdo, wq, at(h_dO, h0 * hb), pq, wq, rows, cudaMemcpyHostToDevice, ds->copy_in)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaEventRecord(ds->ev_in[c], ds->copy_in)) != cudaSuccess) return cuda_fail(e);
+            // compute on the caller's stream; the second half of ALL heads is shifted
+            if ((e = cudaStreamWaitEvent(st, ds->ev_in[c], 0)) != cudaSuccess) return cuda_fail(e);
+            int n_unshifted = H / 2 - h0;
+            n_unshifted = n_unshifted < 0 ? 0 : (n_unshifted > hc ? hc : n_unshifted);
+            const float scale = 1.0f / sqrtf(static_cast<float>(d));
+            int rc2 = fwd_impl(cq, ck, cv, co, cl, B, N, hc, kvc, d, G, scale, n_unshifted, G / 2, 0u, stream, TokStrides());
+            if (rc2 != S2A_OK) return rc2;
+            rc2 = bwd_impl(cq, ck, cv, co, cl, cdo, cdq, cdk, cdv, B, N, hc, kvc, d, G, scale, n_unshifted, G / 2, workspace,
+                           workspace_bytes, stream, kStageAll);
+            if (rc2 != S2A_OK) return rc2;
+            if ((e = cudaEventRecord(ds->ev_compute[c], st)) != cudaSuccess) return cuda_fail(e);
+            // device -> host
+            if ((e = cudaStreamWaitEvent(ds->copy_out, ds->ev_compute[c], 0)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaMemcpy2DAsync(at(h_o, h0 * hb), pq, co, wq, wq, rows, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaMemcpy2DAsync(at(h_lse, static_cast<size_t>(h0) * N * sizeof(float)), pl, cl, wl, wl, B, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaMemcpy2DAsync(at(h_dq, h0 * hb), pq, cdq, wq, wq, rows, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaMemcpy2DAsync(at(h_dk, kv0[c] * hb), pk, cdk, wk, wk, rows, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaMemcpy2DAsync(at(h_dv, kv0[c] * hb), pk, cdv, wk, wk, rows, cudaMemcpyDeviceToHost, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
+        }
+        return S2A_OK;
+    };
+    rc = enqueue_all();
+    // the caller's stream is done when the last copy back is (also after a failure part-way)
+    const int saved_cuda_error = tl_last_cuda_error;
+    const cudaError_t ej = join();
+    if (rc != S2A_OK) {
+        tl_last_cuda_error = saved_cuda_error;
+        return rc;
     }
-    // the caller's stream is done when the last copy back is
-    if ((e = cudaEventRecord(ds->ev_done, ds->copy_out)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaStreamWaitEvent(st, ds->ev_done, 0)) != cudaSuccess) return cuda_fail(e);
-    return S2A_OK;
+    return ej == cudaSuccess ? S2A_OK : cuda_fail(ej);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -475,6 +557,16 @@ int s2a_bwd_noalloc(const void* q, const void* k, const void* v, const void* o, 
 
 size_t s2a_bwd_noalloc_max_rows(void) { return kBuiltinScratchRows; }
 
+int s2a_selftest_wait_expiry(long long limit_cycles, void* stream) {
+    if (limit_cycles < 1 || limit_cycles > kWaitLimitCycles) return S2A_ERR_INVALID_ARG;
+    DeviceState* ds = nullptr;
+    const int rc = prepare_device(&ds);
+    if (rc != S2A_OK) return rc;
+    s2a_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ds->status_ptr, ds->host_word_dev, limit_cycles);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? S2A_OK : cuda_fail(e);
+}
+
 int s2a_device_status(int* where) {
     DeviceState* ds = nullptr;
     int rc = prepare_device(&ds);
@@ -488,6 +580,7 @@ int s2a_device_status(int* where) {
         const int zero = 0;
         e = cudaMemcpy(ds->status_ptr, &zero, sizeof zero, cudaMemcpyHostToDevice);
         if (e != cudaSuccess) return cuda_fail(e);
+        *ds->host_word = 0;
         if (where) *where = word;
         return S2A_ERR_TIMEOUT;
     }

@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(DqCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_slot;
-    const WaitCtx ctx{&bars->abort_flag, p.status};
+    const WaitCtx ctx{&bars->abort_flag, p.status, p.host_status};
     constexpr uint32_t kColAcc = 0, kColS = 128, kColP = 384;
 
     if (warp == 0) {
@@ -586,7 +586,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_slot;
-    const WaitCtx ctx{&bars->abort_flag, p.status};
+    const WaitCtx ctx{&bars->abort_flag, p.status, p.host_status};
     constexpr uint32_t kColDV = 0, kColDK = 128, kColS = 256, kColP = 448;
 
     if (warp == 0) {

@@ -121,7 +121,7 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const WaitCtx ctx{abort_flag, p.status};
+    const WaitCtx ctx{abort_flag, p.status, p.host_status};
 
     if (warp == 0) {
         // =========================== TMA producer ============================================
@@ -239,8 +239,7 @@ __global__ void __launch_bounds__(FwdCfg<HD>::kThreads, 2) s2a_fwd_kernel(const 
                 if ((spins & 255u) == 0) {
                     if (*abort_flag != 0) return false;
                     if (clock64() - t0 > kWaitLimitCycles) {
-                        *abort_flag = kWaitFwd + 9;
-                        atomicCAS(p.status, 0, kWaitFwd + 9);
+                        report_expiry(ctx, kWaitFwd + 9);
                         return false;
                     }
                 }

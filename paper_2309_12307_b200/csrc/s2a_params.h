@@ -114,7 +114,8 @@ struct alignas(64) FwdParams {
     CUtensorMap tm_v;
     __nv_bfloat16* o;
     float* lse;
-    int* status;
+    int* status;       // device status word (see WaitCtx)
+    int* host_status;  // its mirror in mapped host memory
     Geometry geo;
     float scale_log2;  // softmax scale * log2(e)
 };
@@ -128,12 +129,13 @@ struct PreParams {
 
 struct alignas(64) BwdDqParams {
     CUtensorMap tm_q, tm_do;  // box (64, 1, 128, 1): the resident query tile
-    CUtensorMap tm_k, tm_v;   // box (64, 1,  64, 1): streamed key sub-tiles
+    CUtensorMap tm_k, tm_v;   // box (64, 1, 128, 1): streamed key tiles
     const float* lse;         // [B, H, N]
     const float* Dsum;        // [B, H, N]
     __nv_bfloat16* dq;
     long long dq_tok_stride;  // elements between consecutive tokens of dq (H * d when dense)
-    int* status;
+    int* status;       // device status word (see WaitCtx)
+    int* host_status;  // its mirror in mapped host memory
     Geometry geo;
     float scale, scale_log2;
 };
@@ -146,7 +148,8 @@ struct alignas(64) BwdDkDvParams {
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
     long long dkv_tok_stride;  // elements between consecutive tokens of dk and dv (Hkv * d when dense)
-    int* status;
+    int* status;       // device status word (see WaitCtx)
+    int* host_status;  // its mirror in mapped host memory
     Geometry geo;
     float scale, scale_log2;
 };

@@ -25,9 +25,6 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
-__device__ __forceinline__ void fence_proxy_async_smem() {
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                  : "memory");
@@ -51,30 +48,45 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 
 // Where bounded waits report: `abort_flag` lives in the CTA's shared memory (non-zero = this CTA is
 // giving up), `status` is the device-wide status word (0 = fine, otherwise the code of the first
-// wait that expired).
+// wait that expired), `host_status` its mirror in mapped host memory, which the host entry points
+// read without synchronising.
 struct WaitCtx {
     volatile int* abort_flag;
     int* status;
+    volatile int* host_status;
 };
 
+// Record that the wait `where` expired: in the CTA's abort flag, in the device status word (first
+// code wins) and in its host-visible mirror.
+__device__ __forceinline__ void report_expiry(const WaitCtx& ctx, int where) {
+    *ctx.abort_flag = where;
+    if (atomicCAS(ctx.status, 0, where) == 0) {
+        *ctx.host_status = where;
+        __threadfence_system();
+    }
+}
+
 // Bounded wait.  Returns false if the CTA is aborting (another thread's wait expired) or if this
-// wait expired; in the latter case it records `where` in the CTA's abort flag and in the device
-// status word.  Callers leave their loop and go to the common teardown.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& ctx, int where) {
+// wait expired (after `limit` SM clock cycles); in the latter case the expiry is reported.
+// Callers leave their loop and go to the common teardown.
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t parity, const WaitCtx& ctx, int where,
+                                                long long limit) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 63u) == 0) {
             if (*ctx.abort_flag != 0) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
-                *ctx.abort_flag = where;
-                atomicCAS(ctx.status, 0, where);
+            if (clock64() - t0 > limit) {
+                report_expiry(ctx, where);
                 return false;
             }
         }
     }
     return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& ctx, int where) {
+    return mbar_wait_limit(bar, parity, ctx, where, kWaitLimitCycles);
 }
 // All 32 lanes wait; the outcome is made warp-uniform so the warp can keep executing warp-wide
 // instructions (or leave its loop) together.
@@ -118,18 +130,6 @@ __device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* t
         ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
-// 4-D tiled store shared -> global (bulk-group completion).
-__device__ __forceinline__ void tma_store_4d(const CUtensorMap* tmap, const void* smem_src, int c0, int c1, int c2,
-                                             int c3) {
-    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(tmap),
-                 "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-                 : "memory");
-}
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read0() {
-    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-}
-__device__ __forceinline__ void tma_store_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // 1-D bulk copy global -> shared (addresses 16-byte aligned, size a multiple of 16 bytes).
 __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -344,11 +344,6 @@ __device__ __forceinline__ uint64_t poly_exp2_x2(uint64_t x2) {
 }
 // Which of the 16 column pairs of a 32-column chunk take poly_exp2_x2 (bit e = pair e): 5 of 16.
 constexpr uint32_t kPolyExpMask = 0x4924u;
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
 // two fp32 -> packed bf16x2 (lo in the low half), round-to-nearest-even
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t r;

@@ -67,3 +67,37 @@ def test_noalloc_rejects_problems_beyond_its_scratch():
     rc = lib.s2a_bwd_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), q.data_ptr(), lse.data_ptr(), dO.data_ptr(),
                              q.data_ptr(), k.data_ptr(), v.data_ptr(), 1, 32768, 32, 32, 128, 8191, None)
     assert rc == s2a.S2A_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("B,N,G,H,Hkv,d", [
+    (1, 32768, 8192, 32, 32, 64),   # B*H*N = 2**20 exactly: the last row of D is the last float of the array
+    (1, 32768, 64, 32, 8, 64),      # the same count with groups smaller than a tile (every tile ragged)
+])
+def test_noalloc_at_exactly_the_limit(B, N, G, H, Hkv, d):
+    """A problem that fills the built-in array to its last element: the statistics of the last query
+    sub-tile are fetched by a bulk copy that ends on the array's last byte.  Bit-equal to s2a_bwd."""
+    from paper_2309_12307_b200 import binding as s2a
+
+    s2a.load()
+    assert B * H * N == s2a.bwd_noalloc_max_rows()
+    q, k, v, dO = (x.cuda() for x in make_inputs(B, N, H, Hkv, d, seed=14))
+    o, lse = s2a.s2a_fwd(q, k, v, G)
+    want = s2a.s2a_bwd(q, k, v, o, lse, dO, G)
+    got = tuple(torch.full_like(x, float("nan")) for x in (q, k, v))
+    s2a.s2a_bwd_noalloc(q, k, v, o, lse, dO, G, *got)
+    torch.cuda.synchronize()
+    assert s2a.device_status() == (0, 0)
+    for name, g, w in zip(("dq", "dk", "dv"), got, want):
+        assert torch.equal(g, w), name
+
+
+def test_noalloc_rejects_four_rows_too_many():
+    from paper_2309_12307_b200 import binding as s2a
+
+    lib = s2a.load()
+    q, k, v, dO = (x.cuda() for x in make_inputs(1, 256, 2, 2, 64, seed=13))
+    lse = torch.zeros((1, 2, 256), dtype=torch.float32, device="cuda")
+    # B*H*N = 2 * 524290 = 2**20 + 4
+    rc = lib.s2a_bwd_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), q.data_ptr(), lse.data_ptr(), dO.data_ptr(),
+                             q.data_ptr(), k.data_ptr(), v.data_ptr(), 1, 524290, 2, 2, 64, 8, None)
+    assert rc == s2a.S2A_ERR_TOO_LARGE

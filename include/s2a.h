@@ -91,16 +91,39 @@ int s2a_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
  *   out: dq, dk, dv (overwritten, not accumulated into)
  *   workspace: caller-owned device scratch of at least s2a_bwd_workspace_bytes(...) bytes,
  *              256-byte aligned; holds D[b,h,t] = dO[b,t,h,:] . o[b,t,h,:] in fp32.
- * dk and dv sum over the H/Hkv query heads that share a KV head inside one thread block, so the
- * result is deterministic (no atomics).  Three kernel launches on `stream`.
+ * dk and dv sum over the H/Hkv query heads that share a KV head inside one thread block, and every dq
+ * row is summed by one thread block in a fixed order, so the results are deterministic (no atomics).
+ *
+ * Two ways to dq, chosen by the size of the workspace alone:
+ *   - minimum workspace: the dq kernel recomputes the scores and dP that the dk/dv kernel also
+ *     computes (14 d multiply-adds per attended pair are executed for the 10 d the derivative needs).
+ *     Three kernel launches on `stream`.
+ *   - a workspace of s2a_bwd_workspace_bytes_fast(...) bytes: the dk/dv kernel also leaves dS (bf16,
+ *     the very values it multiplies with q) in the workspace and dq = scale * dS k is a plain product
+ *     that reads them back: nothing is computed twice, at the price of 2 bytes of scratch per attended
+ *     pair, written once and read once.  If the workspace holds the dS of only some of the KV heads,
+ *     the KV heads are worked off in several passes (two launches and one 4-byte memset per pass).
+ *   dk and dv are bit-identical either way; dq agrees to rounding (the fp32 sums inside the score
+ *   products run in a different order).
  */
 int s2a_bwd(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO,
             void* dq, void* dk, void* dv,
             int B, int N, int H, int Hkv, int d, int G,
             void* workspace, size_t workspace_bytes, void* stream);
 
-/* Bytes of scratch s2a_bwd needs for these sizes (0 if the sizes are invalid). */
+/* Least bytes of scratch s2a_bwd needs for these sizes (0 if the sizes are invalid). */
 size_t s2a_bwd_workspace_bytes(int B, int N, int H, int Hkv, int d, int G);
+
+/*
+ * The workspace size, not above `budget` bytes, with which s2a_bwd and its variants are fastest: the
+ * minimum plus room for the dS of as many whole KV heads (with their H/Hkv query heads) as the budget
+ * allows, all of them if it can: B * H * (N/G) * T * (T+1) * 16 KiB with T = G/128 tiles per group
+ * (one more per run of a group where G/2 is not a multiple of 128).  Returns the minimum size when not
+ * even one KV head fits, 0 if the sizes are invalid.  Any workspace between the two sizes is valid;
+ * what counts is how many KV heads fit.  (The paper has no counterpart: it trains through a library
+ * attention kernel.)
+ */
+size_t s2a_bwd_workspace_bytes_fast(int B, int N, int H, int Hkv, int d, int G, size_t budget);
 
 /*
  * Generalised forms (Section 3.2 pilot study, Table 6 and Appendix B variants 1 and 2): the first
@@ -153,7 +176,7 @@ int s2a_bwd_packed(const void* qkv, const void* o, const float* lse, const void*
  * unpredictable cost of cudaMalloc / cudaFree; a component whose rules forbid allocation after
  * initialisation.  s2a_bwd wants a workspace from such a caller; this variant does not.
  *
- * It computes exactly what s2a_bwd computes (same kernels, same results), but keeps
+ * It computes exactly what s2a_bwd computes with a minimum workspace (same kernels, same results), but keeps
  * D = rowsum(dO * o) in an array that is part of the library image: 2^20 fp32 values (4 MiB) on
  * every GPU that loads the library, held until the process exits.  It calls no allocation routine
  * of any kind.
@@ -181,8 +204,9 @@ size_t s2a_bwd_noalloc_max_rows(void);
  * One kernel of s2a_bwd at a time, for profiling and per-kernel timing: same arguments and
  * semantics as s2a_bwd, but only kernel `stage` is enqueued:
  *   0 = D = rowsum(dO * o) into the workspace, 1 = dk and dv, 2 = dq.
- * Stages 1 and 2 read the workspace stage 0 wrote.  Calling stages 0, 1, 2 in order on one stream
- * is exactly s2a_bwd.
+ * Stages 1 and 2 read the workspace stage 0 wrote (stage 2 also what stage 1 left there, when the
+ * workspace is large enough to hold the dS of ALL KV heads; a smaller one selects the recomputing dq
+ * kernel here).  Calling stages 0, 1, 2 in order on one stream is exactly s2a_bwd with that choice.
  */
 int s2a_bwd_stage(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO,
                   void* dq, void* dk, void* dv,

@@ -23,7 +23,7 @@ S2A_ERR_TIMEOUT = -4
 S2A_ERR_TOO_LARGE = -5
 
 EXPORTS = [
-    "s2a_fwd", "s2a_bwd", "s2a_bwd_workspace_bytes", "s2a_fwd_ex", "s2a_bwd_ex", "s2a_bwd_stage", "s2a_fwd_bwd_host",
+    "s2a_fwd", "s2a_bwd", "s2a_bwd_workspace_bytes", "s2a_bwd_workspace_bytes_fast", "s2a_fwd_ex", "s2a_bwd_ex", "s2a_bwd_stage", "s2a_fwd_bwd_host",
     "s2a_bwd_noalloc", "s2a_bwd_noalloc_max_rows", "s2a_fwd_packed", "s2a_bwd_packed",
     "s2a_selftest_wait_expiry", "s2a_device_status", "s2a_status_string", "s2a_last_cuda_error", "s2a_version",
 ]
@@ -66,6 +66,8 @@ def load() -> ctypes.CDLL:
     lib.s2a_bwd_packed.restype = I
     lib.s2a_bwd_workspace_bytes.argtypes = [I, I, I, I, I, I]
     lib.s2a_bwd_workspace_bytes.restype = Z
+    lib.s2a_bwd_workspace_bytes_fast.argtypes = [I, I, I, I, I, I, Z]
+    lib.s2a_bwd_workspace_bytes_fast.restype = Z
     lib.s2a_fwd_bwd_host.argtypes = [P] * 18 + [I] * 6 + [P, Z, P]
     lib.s2a_fwd_bwd_host.restype = I
     lib.s2a_selftest_wait_expiry.argtypes = [ctypes.c_longlong, P]
@@ -154,7 +156,23 @@ def _check_workspace(ws, device):
 
 
 def bwd_workspace_bytes(B, N, H, Hkv, d, G) -> int:
+    """Least workspace of the backward (dq then recomputes the scores)."""
     return int(load().s2a_bwd_workspace_bytes(B, N, H, Hkv, d, G))
+
+
+def bwd_workspace_bytes_fast(B, N, H, Hkv, d, G, budget: int) -> int:
+    """Workspace, at most `budget` bytes, with which the backward is fastest (room for spilled dS)."""
+    return int(load().s2a_bwd_workspace_bytes_fast(B, N, H, Hkv, d, G, int(budget)))
+
+
+def _default_workspace(B, N, H, Hkv, d, G, device, fast=True):
+    """Workspace for a call that was given none: the fast size within half of the free device memory,
+    or the minimum with fast=False."""
+    need = bwd_workspace_bytes(B, N, H, Hkv, d, G)
+    if fast:
+        free, _ = torch.cuda.mem_get_info(device)
+        need = max(need, bwd_workspace_bytes_fast(B, N, H, Hkv, d, G, free // 2))
+    return torch.empty(max(need, 256), dtype=torch.uint8, device=device)
 
 
 def s2a_fwd(q, k, v, G, o=None, lse=None, stream=None):
@@ -171,16 +189,16 @@ def s2a_fwd(q, k, v, G, o=None, lse=None, stream=None):
     return o, lse
 
 
-def s2a_bwd(q, k, v, o, lse, dO, G, dq=None, dk=None, dv=None, workspace=None, stream=None):
-    """dq, dk, dv (bf16) of sum(o * dO)."""
+def s2a_bwd(q, k, v, o, lse, dO, G, dq=None, dk=None, dv=None, workspace=None, stream=None, fast=True):
+    """dq, dk, dv (bf16) of sum(o * dO).  Without a workspace one is allocated: large enough for the
+    spilling backward (fast=True) or the minimum (fast=False: dq recomputes the scores)."""
     B, N, H, Hkv, d = _dims(q, k, v)
     dq = torch.empty_like(q) if dq is None else dq
     dk = torch.empty_like(k) if dk is None else dk
     dv = torch.empty_like(v) if dv is None else dv
     _check_bwd(q, k, o, lse, dO, dq, dk, dv)
-    need = bwd_workspace_bytes(B, N, H, Hkv, d, G)
     if workspace is None:
-        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+        workspace = _default_workspace(B, N, H, Hkv, d, G, q.device, fast)
     _check_workspace(workspace, q.device)
     rc = load().s2a_bwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), dO.data_ptr(),
                         dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, N, H, Hkv, d, G, workspace.data_ptr(),
@@ -229,7 +247,7 @@ def s2a_fwd_packed(qkv, G, o=None, lse=None, stream=None):
     return o, lse
 
 
-def s2a_bwd_packed(qkv, o, lse, dO, G, dqkv=None, workspace=None, stream=None):
+def s2a_bwd_packed(qkv, o, lse, dO, G, dqkv=None, workspace=None, stream=None, fast=True):
     """Backward on a packed qkv tensor; returns dqkv [B, N, 3, H, d]."""
     B, N, H, d = _packed_dims(qkv)
     dqkv = torch.empty_like(qkv) if dqkv is None else dqkv
@@ -237,9 +255,8 @@ def s2a_bwd_packed(qkv, o, lse, dO, G, dqkv=None, workspace=None, stream=None):
     _require(o, torch.bfloat16, "o", shape=(B, N, H, d), device=qkv.device)
     _require(dO, torch.bfloat16, "dO", shape=(B, N, H, d), device=qkv.device)
     _require(lse, torch.float32, "lse", shape=(B, H, N), device=qkv.device)
-    need = bwd_workspace_bytes(B, N, H, H, d, G)
     if workspace is None:
-        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=qkv.device)
+        workspace = _default_workspace(B, N, H, H, d, G, qkv.device, fast)
     _check_workspace(workspace, qkv.device)
     rc = load().s2a_bwd_packed(qkv.data_ptr(), o.data_ptr(), lse.data_ptr(), dO.data_ptr(), dqkv.data_ptr(), B, N, H, d, G,
                                workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr(stream))
@@ -285,7 +302,7 @@ def s2a_fwd_ex(q, k, v, G, scale=None, n_unshifted=None, shift=None, leak_free=F
 
 
 def s2a_bwd_ex(q, k, v, o, lse, dO, G, scale=None, n_unshifted=None, shift=None, leak_free=False, workspace=None,
-               stream=None, dq=None, dk=None, dv=None, swap_wrapped=False):
+               stream=None, dq=None, dk=None, dv=None, swap_wrapped=False, fast=True):
     B, N, H, Hkv, d = _dims(q, k, v)
     scale = 1.0 / math.sqrt(d) if scale is None else scale
     n_unshifted = H // 2 if n_unshifted is None else n_unshifted
@@ -294,9 +311,8 @@ def s2a_bwd_ex(q, k, v, o, lse, dO, G, scale=None, n_unshifted=None, shift=None,
     dk = torch.empty_like(k) if dk is None else dk
     dv = torch.empty_like(v) if dv is None else dv
     _check_bwd(q, k, o, lse, dO, dq, dk, dv)
-    need = bwd_workspace_bytes(B, N, H, Hkv, d, G)
     if workspace is None:
-        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+        workspace = _default_workspace(B, N, H, Hkv, d, G, q.device, fast)
     _check_workspace(workspace, q.device)
     rc = load().s2a_bwd_ex(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), dO.data_ptr(),
                            dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), B, N, H, Hkv, d, G, scale, n_unshifted, shift,

@@ -37,6 +37,7 @@ struct DeviceState {
     int* status_ptr = nullptr;        // device address of g_status_word
     volatile int* host_word = nullptr;  // this device's mirror, host address
     int* host_word_dev = nullptr;     // the same word as the device sees it
+    int n_sm = 0;                     // multiprocessors (grid of the persistent kernel)
     // s2a_fwd_bwd_host only: copy streams and the events that order them against the caller's stream
     bool host_path_ready = false;
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
@@ -70,6 +71,8 @@ int prepare_device(DeviceState** out) {
         e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
         if (e != cudaSuccess) return cuda_fail(e);
         if (major != 10) return S2A_ERR_UNSUPPORTED;
+        e = cudaDeviceGetAttribute(&ds.n_sm, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_fail(e);
         if (!g_encode) {
             void* fn = nullptr;
             cudaDriverEntryPointQueryResult qres;
@@ -281,12 +284,35 @@ size_t s2a_bwd_workspace_bytes(int B, int N, int H, int Hkv, int d, int G) {
 }
 
 namespace {
+// Workspace layout: D [B, H, N] fp32 (the minimum), then 256 bytes of counters, then the spill area.
+constexpr size_t kSpillHeaderBytes = 256;
+constexpr size_t kSpillBlockBytes = static_cast<size_t>(kSpillBlockElems) * 2;
+// spill blocks of one KV head with its query heads, for groups of at most T tiles
+size_t spill_blocks_per_kv_head(int B, int N, int H, int Hkv, int G, int T) {
+    return static_cast<size_t>(B) * (H / Hkv) * (N / G) * static_cast<size_t>(spill_blocks_per_unit(T));
+}
+}  // namespace
+
+size_t s2a_bwd_workspace_bytes_fast(int B, int N, int H, int Hkv, int d, int G, size_t budget) {
+    const size_t min_bytes = s2a_bwd_workspace_bytes(B, N, H, Hkv, d, G);
+    if (min_bytes == 0) return 0;
+    // tiles of the largest group: G / 128 when G and the default shift G / 2 are multiples of the tile,
+    // otherwise one partial tile per run of the group that wraps
+    const int T = (G % (2 * kTile) == 0) ? G / kTile : (G + kTile - 1) / kTile + 1;
+    const size_t per_kv = spill_blocks_per_kv_head(B, N, H, Hkv, G, T) * kSpillBlockBytes;
+    if (budget <= min_bytes + kSpillHeaderBytes) return min_bytes;
+    size_t nk = (budget - min_bytes - kSpillHeaderBytes) / per_kv;
+    if (nk > static_cast<size_t>(Hkv)) nk = Hkv;
+    return nk == 0 ? min_bytes : min_bytes + kSpillHeaderBytes + nk * per_kv;
+}
+
+namespace {
 enum : unsigned { kStagePre = 1u, kStageDkDv = 2u, kStageDq = 4u, kStageAll = 7u };
 
 int bwd_impl(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO, void* dq,
              void* dk, void* dv, int B, int N, int H, int Hkv, int d, int G, float scale, int n_unshifted, int shift,
              void* workspace, size_t workspace_bytes, void* stream, unsigned stages, unsigned flags = 0u,
-             const TokStrides& ts = TokStrides()) {
+             const TokStrides& ts = TokStrides(), bool may_spill = true) {
     if (!q || !k || !v || !o || !lse || !dO || !dq || !dk || !dv || !workspace) return S2A_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse) || !aligned16(dO) ||
         !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
@@ -324,23 +350,65 @@ int bwd_impl(const void* q, const void* k, const void* v, const void* o, const f
     pk.lse = lse, pk.Dsum = Dsum;
     pk.dk = static_cast<__nv_bfloat16*>(dk), pk.dv = static_cast<__nv_bfloat16*>(dv);
     pk.status = ds->status_ptr, pk.host_status = ds->host_word_dev, pk.geo = geo, pk.scale = scale, pk.scale_log2 = scale * kLog2eHost;
+    pk.spill = nullptr;
+    pk.pass.hk0 = 0, pk.pass.nk = Hkv;
 
     PreParams pp;
     pp.o = static_cast<const __nv_bfloat16*>(o), pp.dO = static_cast<const __nv_bfloat16*>(dO), pp.Dsum = Dsum;
     pp.B = B, pp.N = N, pp.H = H;
+
+    // How many KV heads' worth of dS^T the workspace can hold beyond D: with room for at least one, the
+    // dK,dV kernel spills dS^T and dQ is a plain product (several passes over the KV heads if they do
+    // not all fit); otherwise dQ recomputes S and dP.  A single-stage call spills only in one pass, so
+    // that stages 0, 1, 2 in order stay equal to the whole backward.
+    const size_t min_bytes = s2a_bwd_workspace_bytes(B, N, H, Hkv, d, G);
+    const size_t per_kv = spill_blocks_per_kv_head(B, N, H, Hkv, G, geo.tiles_per_group);
+    size_t nk_fit = 0;
+    if (may_spill && workspace_bytes > min_bytes + kSpillHeaderBytes)
+        nk_fit = (workspace_bytes - min_bytes - kSpillHeaderBytes) / (per_kv * kSpillBlockBytes);
+    if (nk_fit > static_cast<size_t>(Hkv)) nk_fit = Hkv;
+    if (stages != kStageAll && nk_fit < static_cast<size_t>(Hkv)) nk_fit = 0;
 
     cudaError_t e;
     if (stages & kStagePre) {
         e = launch_bwd_preprocess(pp, d, st);
         if (e != cudaSuccess) return cuda_fail(e);
     }
-    if (stages & kStageDkDv) {
-        e = launch_bwd_dkdv(pk, d, st);
-        if (e != cudaSuccess) return cuda_fail(e);
+    if (nk_fit == 0) {
+        if (stages & kStageDkDv) {
+            e = launch_bwd_dkdv(pk, d, st);
+            if (e != cudaSuccess) return cuda_fail(e);
+        }
+        if (stages & kStageDq) {
+            e = launch_bwd_dq(pq, d, st);
+            if (e != cudaSuccess) return cuda_fail(e);
+        }
+        return S2A_OK;
     }
-    if (stages & kStageDq) {
-        e = launch_bwd_dq(pq, d, st);
-        if (e != cudaSuccess) return cuda_fail(e);
+
+    char* base = static_cast<char*>(workspace);
+    int* counter = reinterpret_cast<int*>(base + min_bytes);
+    pk.spill = reinterpret_cast<__nv_bfloat16*>(base + min_bytes + kSpillHeaderBytes);
+    BwdDqSpillParams ps;
+    memset(&ps, 0, sizeof ps);
+    ps.tm_k = pq.tm_k;
+    ps.spill = pk.spill;
+    ps.dq = pq.dq, ps.dq_tok_stride = pq.dq_tok_stride, ps.counter = counter;
+    ps.status = ds->status_ptr, ps.host_status = ds->host_word_dev, ps.geo = geo, ps.scale = scale;
+    for (int hk0 = 0; hk0 < Hkv; hk0 += static_cast<int>(nk_fit)) {
+        const int nk = Hkv - hk0 < static_cast<int>(nk_fit) ? Hkv - hk0 : static_cast<int>(nk_fit);
+        pk.pass.hk0 = hk0, pk.pass.nk = nk;
+        ps.pass = pk.pass;
+        if (stages & kStageDkDv) {
+            e = launch_bwd_dkdv(pk, d, st);
+            if (e != cudaSuccess) return cuda_fail(e);
+        }
+        if (stages & kStageDq) {
+            e = cudaMemsetAsync(counter, 0, sizeof(int), st);
+            if (e != cudaSuccess) return cuda_fail(e);
+            e = launch_bwd_dq_spill(ps, d, ds->n_sm, st);
+            if (e != cudaSuccess) return cuda_fail(e);
+        }
     }
     return S2A_OK;
 }
@@ -552,7 +620,7 @@ int s2a_bwd_noalloc(const void* q, const void* k, const void* v, const void* o, 
     // Every row of D that the two gradient kernels read is rewritten by the first kernel of this
     // call, so nothing left in the array by an earlier call has to be cleared.
     return bwd_impl(q, k, v, o, lse, dO, dq, dk, dv, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2,
-                    G / 2, scratch, kBuiltinScratchRows * sizeof(float), stream, kStageAll);
+                    G / 2, scratch, kBuiltinScratchRows * sizeof(float), stream, kStageAll, 0u, TokStrides(), false);
 }
 
 size_t s2a_bwd_noalloc_max_rows(void) { return kBuiltinScratchRows; }

@@ -494,13 +494,14 @@ __global__ void __launch_bounds__(DqCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(cons
 // key tile is a tile of every head's partition.)
 struct HeadWalk {
     GroupLayout L;
-    int j, n_begin, n_end;
+    int g, j, n_begin, n_end;
 };
 __device__ __forceinline__ HeadWalk head_walk(const Geometry& geo, int hq, int tk0) {
     HeadWalk w;
     const int s = (hq < geo.n_unshifted) ? 0 : geo.shift;
     const int pos = mod_pos(tk0 - s, geo.N);
-    w.L = group_layout(geo, s, pos / geo.G);
+    w.g = pos / geo.G;
+    w.L = group_layout(geo, s, w.g);
     const int in_group = pos % geo.G;
     const int nB = w.L.nTiles - w.L.nA;
     w.j = in_group < w.L.lenA ? (w.L.swapped ? nB : 0) + in_group / kTile
@@ -510,7 +511,8 @@ __device__ __forceinline__ HeadWalk head_walk(const Geometry& geo, int hq, int t
     return w;
 }
 
-template <int HD>
+// kSpill: every step's dS^T also goes to global memory (see SpillPass) for s2a_bwd_dq_spill_kernel.
+template <int HD, bool kSpill>
 __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(const __grid_constant__ BwdDkDvParams p) {
     using C = BwdCfg<HD>;
     using Bars = BwdBars<C::kStages>;
@@ -539,10 +541,10 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
     // (earliest in the group) first
     const int Tg = geo.tiles_per_group;
     int unit, j0;
-    decode_block(blockIdx.x, geo.B * geo.Hkv * geo.groups, Tg, &unit, &j0);
+    decode_block(blockIdx.x, geo.B * p.pass.nk * geo.groups, Tg, &unit, &j0);
     const int g0 = unit % geo.groups;
-    const int hk = (unit / geo.groups) % geo.Hkv;
-    const int b = unit / (geo.groups * geo.Hkv);
+    const int hk = p.pass.hk0 + (unit / geo.groups) % p.pass.nk;
+    const int b = unit / (geo.groups * p.pass.nk);
     const int hq0 = hk * rep;
     const int s0 = (hq0 < geo.n_unshifted) ? 0 : geo.shift;
     const GroupLayout L0 = group_layout(geo, s0, g0);
@@ -716,10 +718,20 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         const int row = quad * 32 + lane;  // key row of the tile owned by this thread
         const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
         const float c2 = p.scale_log2;
+        const bool key_valid = row < tk.valid;  // rows past the end of a ragged tile belong to other tiles
         bool ok = true;
         int it = 0;
         for (int hq = hq0; ok && hq < hq0 + rep; ++hq) {
             const HeadWalk w = head_walk(geo, hq, tk0);
+            // where this thread's 32 dS^T values of a step (four 16-byte chunks) go when they are spilled:
+            // chunks 4 half .. 4 half + 3 of key row `row` in block (j, n) of the spill unit (b, hq, g).  A
+            // block is stored chunk-major, so the 32 lanes of a warp write 512 contiguous bytes at a time.
+            uint4* spill_dst = nullptr;
+            if constexpr (kSpill) {
+                const long long su = (static_cast<long long>(b) * (p.pass.nk * rep) + (hq - p.pass.hk0 * rep)) * geo.groups + w.g;
+                spill_dst = reinterpret_cast<uint4*>(p.spill + spill_block(su, Tg, w.j, w.n_begin) * kSpillBlockElems) +
+                            half * 4 * kTile + row;
+            }
             for (int n = w.n_begin; n < w.n_end; ++n, ++it) {
                 const int st = it % C::kStages;
                 const int bf = it % kBufs;
@@ -807,6 +819,16 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                 }
                 tmem_st_32x16(tS, pkP);
                 tmem_st_32x16(tS + 16, pkS);
+                if constexpr (kSpill) {
+                    // streaming stores: written once, read once by the dQ kernel much later
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint4 x = make_uint4(pkS[4 * c], pkS[4 * c + 1], pkS[4 * c + 2], pkS[4 * c + 3]);
+                        if (!key_valid) x = make_uint4(0u, 0u, 0u, 0u);
+                        __stcs(spill_dst + c * kTile, x);
+                    }
+                    spill_dst += kSpillBlockElems * 2 / sizeof(uint4);
+                }
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(&bars->p_full[bf]);
@@ -815,15 +837,245 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDkDv + 7)) {
             tc_fence_after();
             const size_t out_row = (static_cast<size_t>(b) * geo.N + tk0 + row) * p.dkv_tok_stride + static_cast<size_t>(hk) * HD;
-            const bool row_valid = row < tk.valid;  // rows past the end of a ragged tile belong to other tiles
-            if (half == 0) store_acc_cols<HD>(t_row + kColDV, 1.0f, p.dv + out_row, row_valid);
-            else store_acc_cols<HD>(t_row + kColDK, p.scale, p.dk + out_row, row_valid);
+            if (half == 0) store_acc_cols<HD>(t_row + kColDV, 1.0f, p.dv + out_row, key_valid);
+            else store_acc_cols<HD>(t_row + kColDK, p.scale, p.dk + out_row, key_valid);
         }
     }
 
     tc_fence_before();
     __syncthreads();
     if (warp == 3) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, C::kTmemCols);
+    }
+}
+
+
+// ------------------------------------------------------------------------------------------------
+// 4. dQ from spilled dS^T
+// ------------------------------------------------------------------------------------------------
+// dQ_i = scale * sum_j dS_ij K_j over the key tiles j_begin..i of the group, with dS_ij read back from
+// the blocks the spilling dK,dV kernel wrote: nothing is recomputed, the kernel is a chain of
+// 128x128x128 products whose A operand streams from global memory once (memory bound).
+//
+// Persistent: one CTA per SM takes (unit, query tile) work items, heaviest first, from a counter in
+// global memory.  Warp 0 draws the items and loads with TMA (it runs ahead across item boundaries, so
+// the ring never drains between items), warp 1 issues the MMAs into one of two accumulators in tensor
+// memory, warps 2-5 write the finished accumulator out while the next item is being multiplied.
+// A block (j, n) is copied to shared memory as it lies in global memory (one bulk copy for the blocks
+// (j, 2i) and (j, 2i+1), which are neighbours): chunk-major, i.e. the 16-byte chunk c (8 queries) of
+// key row r at byte (c * 128 + r) * 16.  Eight key rows of one chunk are 128 contiguous bytes: the
+// "core matrix" of an MN-major operand without swizzle (M = queries, K = keys), with 2048 bytes
+// between chunks along M and 128 bytes between groups of 8 keys along K; the two blocks side by side
+// are the 128-query A operand.  B is the K tile, MN-major (N = d) with the 128-byte swizzle TMA
+// leaves, as in the recomputing dQ kernel.
+template <int HD>
+struct DqSpillCfg {
+    static constexpr int kThreads = 192;  // TMA warp, MMA warp, four epilogue warps
+    static constexpr int kBoxes = HD / 64;
+    static constexpr int kKBoxBytes = kTile * 128;
+    static constexpr int kKBytes = kBoxes * kKBoxBytes;
+    static constexpr int kDsBlockBytes = kSpillBlockElems * 2;
+    static constexpr int kStageBytes = 2 * kDsBlockBytes + kKBytes;
+    static constexpr int kStages = 3;
+    static constexpr int kSched = 8;  // work items the producer can be ahead of the epilogue: at most 5
+    static constexpr int kBarBytes = 512;
+    static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kBarBytes;
+    static constexpr int kTmemCols = 256;  // two accumulators of 128 columns
+};
+
+struct DqSpillBars {
+    uint64_t full[3], empty[3];
+    uint64_t acc_full[2], acc_empty[2];
+    uint64_t sched_full[8];
+    uint64_t drain;
+    long long item[8];
+    uint32_t tmem_slot;
+    int abort_flag;
+};
+
+struct DqSpillItem {
+    int b, h, hk, i, j_begin, n_steps, tq0, q_valid;
+    long long unit;
+    GroupLayout L;
+};
+// Work item `id` (heaviest query tiles of a chunk of units first, as in the other kernels).  n_steps = 0
+// marks a slot of a group that has fewer tiles than the largest one.
+__device__ __forceinline__ DqSpillItem dq_spill_item(const Geometry& geo, const SpillPass& pass, long long id) {
+    DqSpillItem t;
+    const int rep = geo.H / geo.Hkv;
+    const int heads = pass.nk * rep;
+    int unit, rank;
+    decode_block(id, geo.B * heads * geo.groups, geo.tiles_per_group, &unit, &rank);
+    const int g = unit % geo.groups;
+    t.h = pass.hk0 * rep + (unit / geo.groups) % heads;
+    t.b = unit / (geo.groups * heads);
+    t.hk = t.h / rep;
+    t.unit = unit;
+    const int s = (t.h < geo.n_unshifted) ? 0 : geo.shift;
+    t.L = group_layout(geo, s, g);
+    t.i = t.L.nTiles - 1 - rank;
+    if (t.i < 0) {
+        t.n_steps = 0;
+        t.j_begin = 0, t.tq0 = 0, t.q_valid = 0;
+        return t;
+    }
+    t.j_begin = first_key_tile(t.L, t.i);
+    t.n_steps = t.i + 1 - t.j_begin;
+    const TileRef tq = tile_ref(t.L, t.i);
+    t.tq0 = tq.tok0;
+    t.q_valid = tq.valid;
+    return t;
+}
+
+template <int HD>
+__global__ void __launch_bounds__(DqSpillCfg<HD>::kThreads, 1) s2a_bwd_dq_spill_kernel(const __grid_constant__ BwdDqSpillParams p) {
+    using C = DqSpillCfg<HD>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    DqSpillBars* bars = reinterpret_cast<DqSpillBars*>(smem + C::kStages * C::kStageBytes);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    __shared__ int s_poisoned;
+    if (threadIdx.x == 0) s_poisoned = *reinterpret_cast<volatile int*>(p.status);
+    __syncthreads();
+    if (s_poisoned != 0) return;
+    const Geometry& geo = p.geo;
+    const int Tg = geo.tiles_per_group;
+    const long long n_items = static_cast<long long>(geo.B) * p.pass.nk * (geo.H / geo.Hkv) * geo.groups * Tg;
+
+    if (threadIdx.x == 0) {
+        for (int x = 0; x < C::kStages; ++x) {
+            mbar_init(&bars->full[x], 1);
+            mbar_init(&bars->empty[x], 1);
+        }
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(&bars->acc_full[x], 1);
+            mbar_init(&bars->acc_empty[x], 128);
+        }
+        for (int x = 0; x < C::kSched; ++x) mbar_init(&bars->sched_full[x], 1);
+        mbar_init(&bars->drain, 1);
+        bars->abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&p.tm_k);
+    }
+    if (warp == 1) {
+        tmem_alloc(&bars->tmem_slot, C::kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = bars->tmem_slot;
+    const WaitCtx ctx{&bars->abort_flag, p.status, p.host_status};
+
+    if (warp == 0) {
+        // ---- scheduler + TMA producer -------------------------------------------------------------
+        if (lane == 0) {
+            long long it = 0;  // stage uses so far
+            bool ok = true;
+            for (int k = 0; ok; ++k) {
+                // draw the next item that has work (slots of groups with fewer tiles than the largest are
+                // skipped here, so the other warps only ever see real items and the end marker)
+                long long id;
+                DqSpillItem t;
+                do {
+                    id = static_cast<long long>(atomicAdd(p.counter, 1));
+                    if (id >= n_items) break;
+                    t = dq_spill_item(geo, p.pass, id);
+                } while (t.n_steps == 0);
+                bars->item[k % C::kSched] = id;
+                mbar_arrive(&bars->sched_full[k % C::kSched]);  // release: the id is visible to whoever sees the phase
+                if (id >= n_items) break;
+                for (int n = 0; n < t.n_steps; ++n, ++it) {
+                    const int st = static_cast<int>(it % C::kStages);
+                    const uint32_t ph = static_cast<uint32_t>(it / C::kStages) & 1u;
+                    if (!mbar_wait(&bars->empty[st], ph ^ 1, ctx, kWaitBwdDqSpill + 1)) { ok = false; break; }
+                    const int j = t.j_begin + n;
+                    uint8_t* sDs = smem + st * C::kStageBytes;
+                    uint8_t* sK = sDs + 2 * C::kDsBlockBytes;
+                    mbar_expect_tx(&bars->full[st], C::kStageBytes);
+                    const long long blk = spill_block(t.unit, Tg, j, 2 * t.i);
+                    bulk_load_1d(sDs, p.spill + blk * kSpillBlockElems, 2 * C::kDsBlockBytes, &bars->full[st]);
+                    const int tk0 = tile_ref(t.L, j).tok0;
+                    for (int bx = 0; bx < C::kBoxes; ++bx)
+                        tma_load_4d(sK + bx * C::kKBoxBytes, &p.tm_k, &bars->full[st], bx * 64, t.hk, tk0, t.b);
+                }
+            }
+            if (bars->abort_flag != 0) {
+                for (long long nn = (it > C::kStages ? it - C::kStages : 0); nn < it; ++nn)
+                    mbar_wait_drain(&bars->full[nn % C::kStages], static_cast<uint32_t>(nn / C::kStages) & 1u);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---- MMA issuer (warp-uniform loop, one elected lane issues) ------------------------------
+        constexpr uint32_t idesc = idesc_bf16(128, HD, 1, 1);
+        long long it = 0;
+        bool ok = true;
+        int used = 0;  // accumulator uses so far
+        for (int k = 0; ok; ++k) {
+            if (!mbar_wait_uniform(&bars->sched_full[k % C::kSched], (k / C::kSched) & 1, ctx, kWaitBwdDqSpill + 2)) break;
+            const long long id = bars->item[k % C::kSched];
+            if (id >= n_items) break;
+            const DqSpillItem t = dq_spill_item(geo, p.pass, id);
+            const int buf = used & 1;
+            if (!mbar_wait_uniform(&bars->acc_empty[buf], ((used >> 1) & 1) ^ 1, ctx, kWaitBwdDqSpill + 3)) break;
+            tc_fence_after();
+            const uint32_t tAcc = tmem_base + buf * 128;
+            for (int n = 0; n < t.n_steps; ++n, ++it) {
+                const int st = static_cast<int>(it % C::kStages);
+                if (!mbar_wait_uniform(&bars->full[st], static_cast<uint32_t>(it / C::kStages) & 1u, ctx, kWaitBwdDqSpill + 4)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t aDs = smem_u32(smem + st * C::kStageBytes);
+                const uint32_t dA = desc_lo_mn_major_plain(aDs, 128);
+                const uint32_t dB = desc_lo_mn_major(aDs + 2 * C::kDsBlockBytes, C::kKBoxBytes);
+                if (elect_one()) {
+#pragma unroll
+                    for (int kk = 0; kk < kTile / 16; ++kk)
+                        mma_ss_hi(tAcc, dA + kk * (256u >> 4), desc_hi_plain(2048), dB + kk * kDescStepMn, kDescHi, idesc,
+                                  (n > 0) || (kk > 0));
+                    mma_commit(&bars->empty[st]);
+                    if (n == t.n_steps - 1) mma_commit(&bars->acc_full[buf]);
+                }
+                __syncwarp();
+            }
+            ++used;
+        }
+        if (__any_sync(0xffffffffu, bars->abort_flag != 0)) {
+            if (elect_one()) {
+                mma_commit(&bars->drain);
+                mbar_wait_drain(&bars->drain, 0);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---- epilogue: thread owns accumulator row 32 * quad + lane -------------------------------
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+        int used = 0;
+        for (int k = 0;; ++k) {
+            if (!mbar_wait(&bars->sched_full[k % C::kSched], (k / C::kSched) & 1, ctx, kWaitBwdDqSpill + 5)) break;
+            const long long id = bars->item[k % C::kSched];
+            if (id >= n_items) break;
+            const DqSpillItem t = dq_spill_item(geo, p.pass, id);
+            const int buf = used & 1;
+            if (!mbar_wait(&bars->acc_full[buf], (used >> 1) & 1, ctx, kWaitBwdDqSpill + 6)) break;
+            tc_fence_after();
+            __nv_bfloat16* dst = p.dq + (static_cast<size_t>(t.b) * geo.N + t.tq0 + row) * p.dq_tok_stride + static_cast<size_t>(t.h) * HD;
+            store_acc_cols<HD>(t_row + buf * 128, p.scale, dst, row < t.q_valid);
+            tc_fence_before();
+            mbar_arrive(&bars->acc_empty[buf]);
+            ++used;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, C::kTmemCols);
     }
@@ -837,10 +1089,18 @@ cudaError_t configure_bwd() {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(s2a_bwd_dq_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqCfg<128>::kSmemBytes);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(s2a_bwd_dkdv_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes);
+    e = cudaFuncSetAttribute(s2a_bwd_dkdv_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(s2a_bwd_dkdv_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                BwdCfg<128>::kSmemBytes);
+    e = cudaFuncSetAttribute(s2a_bwd_dkdv_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<128>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(s2a_bwd_dkdv_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<64>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(s2a_bwd_dkdv_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<128>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(s2a_bwd_dq_spill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSpillCfg<64>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(s2a_bwd_dq_spill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                DqSpillCfg<128>::kSmemBytes);
 }
 
 cudaError_t launch_bwd_preprocess(const PreParams& p, int d, cudaStream_t stream) {
@@ -861,9 +1121,23 @@ cudaError_t launch_bwd_dq(const BwdDqParams& p, int d, cudaStream_t stream) {
 
 cudaError_t launch_bwd_dkdv(const BwdDkDvParams& p, int d, cudaStream_t stream) {
     const Geometry& g = p.geo;
-    const unsigned grid = static_cast<unsigned>(static_cast<long long>(g.B) * g.Hkv * g.groups * g.tiles_per_group);
-    if (d == 64) s2a_bwd_dkdv_kernel<64><<<grid, BwdCfg<64>::kThreads, BwdCfg<64>::kSmemBytes, stream>>>(p);
-    else s2a_bwd_dkdv_kernel<128><<<grid, BwdCfg<128>::kThreads, BwdCfg<128>::kSmemBytes, stream>>>(p);
+    const unsigned grid = static_cast<unsigned>(static_cast<long long>(g.B) * p.pass.nk * g.groups * g.tiles_per_group);
+    if (p.spill != nullptr) {
+        if (d == 64) s2a_bwd_dkdv_kernel<64, true><<<grid, BwdCfg<64>::kThreads, BwdCfg<64>::kSmemBytes, stream>>>(p);
+        else s2a_bwd_dkdv_kernel<128, true><<<grid, BwdCfg<128>::kThreads, BwdCfg<128>::kSmemBytes, stream>>>(p);
+    } else {
+        if (d == 64) s2a_bwd_dkdv_kernel<64, false><<<grid, BwdCfg<64>::kThreads, BwdCfg<64>::kSmemBytes, stream>>>(p);
+        else s2a_bwd_dkdv_kernel<128, false><<<grid, BwdCfg<128>::kThreads, BwdCfg<128>::kSmemBytes, stream>>>(p);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_bwd_dq_spill(const BwdDqSpillParams& p, int d, int n_sm, cudaStream_t stream) {
+    const Geometry& g = p.geo;
+    const long long items = static_cast<long long>(g.B) * p.pass.nk * (g.H / g.Hkv) * g.groups * g.tiles_per_group;
+    const unsigned grid = static_cast<unsigned>(items < n_sm ? items : n_sm);
+    if (d == 64) s2a_bwd_dq_spill_kernel<64><<<grid, DqSpillCfg<64>::kThreads, DqSpillCfg<64>::kSmemBytes, stream>>>(p);
+    else s2a_bwd_dq_spill_kernel<128><<<grid, DqSpillCfg<128>::kThreads, DqSpillCfg<128>::kSmemBytes, stream>>>(p);
     return cudaGetLastError();
 }
 

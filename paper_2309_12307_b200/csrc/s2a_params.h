@@ -16,6 +16,7 @@ enum WaitCode : int {
     kWaitFwd = 100,
     kWaitBwdDq = 200,
     kWaitBwdDkDv = 300,
+    kWaitBwdDqSpill = 400,
 };
 
 // Block order shared by the tensor-core kernels.  A "unit" is one (batch, head, group); it has
@@ -140,6 +141,24 @@ struct alignas(64) BwdDqParams {
     float scale, scale_log2;
 };
 
+// The dK,dV kernel can leave its dS^T values (bf16) in global memory for a dQ kernel that then only
+// has to multiply them with K instead of recomputing S and dP.  One pass covers the KV heads
+// [hk0, hk0 + nk) with their query heads; a "spill unit" is one (batch, query head of the pass, group),
+// numbered (b * nk * rep + (hq - hk0 * rep)) * groups + g.  A unit owns T (T + 1) blocks, T =
+// tiles_per_group: block (j, n) holds dS^T of key tile j and 64-query sub-tile n >= 2 j, 128 key rows of
+// 64 bf16 (16 KB), stored chunk-major: the 16-byte chunk c (queries 8 c .. 8 c + 7) of key row r sits at
+// byte (c * 128 + r) * 16 of the block, which is both what a warp of the dK,dV kernel writes in one
+// coalesced store and an operand layout the tensor core reads directly.  Masked entries and rows that
+// are not part of the group are zero.
+struct SpillPass {
+    int hk0, nk;  // KV heads of this pass
+};
+__host__ __device__ inline long long spill_blocks_per_unit(int T) { return static_cast<long long>(T) * (T + 1); }
+__host__ __device__ inline long long spill_block(long long unit, int T, int j, int n) {
+    return unit * spill_blocks_per_unit(T) + static_cast<long long>(j) * (2 * T - j + 1) + (n - 2 * j);
+}
+constexpr int kSpillBlockElems = kTile * kSubTile;  // bf16 values per block
+
 struct alignas(64) BwdDkDvParams {
     CUtensorMap tm_k, tm_v;   // box (64, 1, 128, 1): the resident key tile
     CUtensorMap tm_q, tm_do;  // box (64, 1,  64, 1): streamed query sub-tiles
@@ -148,17 +167,34 @@ struct alignas(64) BwdDkDvParams {
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
     long long dkv_tok_stride;  // elements between consecutive tokens of dk and dv (Hkv * d when dense)
+    __nv_bfloat16* spill;      // dS^T blocks of this pass (spilling variant only)
+    SpillPass pass;            // KV heads this launch covers (all of them when nothing is spilled)
     int* status;       // device status word (see WaitCtx)
     int* host_status;  // its mirror in mapped host memory
     Geometry geo;
     float scale, scale_log2;
 };
 
+// dQ from spilled dS^T: dQ_i = scale * sum_j dS_ij K_j, one CTA per 128-query tile.
+struct alignas(64) BwdDqSpillParams {
+    CUtensorMap tm_k;   // box (64, 1, 128, 1): streamed key tiles
+    const __nv_bfloat16* spill;  // the blocks the dK,dV kernel of this pass wrote
+    __nv_bfloat16* dq;
+    long long dq_tok_stride;
+    int* counter;  // next work item; zero when the kernel starts
+    SpillPass pass;
+    int* status;
+    int* host_status;
+    Geometry geo;
+    float scale;
+};
+
 // Enqueue one kernel each on `stream`; return the launch error, if any.
 cudaError_t launch_fwd(const FwdParams& p, int d, cudaStream_t stream);
 cudaError_t launch_bwd_preprocess(const PreParams& p, int d, cudaStream_t stream);
 cudaError_t launch_bwd_dq(const BwdDqParams& p, int d, cudaStream_t stream);
-cudaError_t launch_bwd_dkdv(const BwdDkDvParams& p, int d, cudaStream_t stream);
+cudaError_t launch_bwd_dkdv(const BwdDkDvParams& p, int d, cudaStream_t stream);  // p.spill != nullptr: spilling variant
+cudaError_t launch_bwd_dq_spill(const BwdDqSpillParams& p, int d, int n_sm, cudaStream_t stream);  // persistent: one CTA per SM
 
 // Per-device kernel attribute set-up (dynamic shared memory sizes).
 cudaError_t configure_fwd();

@@ -130,6 +130,13 @@ __device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* t
         ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
+// 2-D tiled load global -> shared (c0 = innermost coordinate, c0 * element size a multiple of 16 B).
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* tmap, uint64_t* bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+        : "memory");
+}
 // 1-D bulk copy global -> shared (addresses 16-byte aligned, size a multiple of 16 bytes).
 __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -227,6 +234,15 @@ __device__ __forceinline__ uint32_t desc_lo_mn_major(uint32_t saddr, uint32_t bl
     return ((saddr & 0x3FFFFu) >> 4) | (((block_stride_bytes >> 4) & 0x3FFFu) << 16);
 }
 constexpr uint32_t kDescStepMn = 2048u >> 4;
+// MN-major operand WITHOUT swizzle: 8 K rows of one 16-byte chunk (8 values of the M/N index) are 128
+// contiguous bytes; `k_group_bytes` separates consecutive groups of 8 K rows (low word, leading
+// offset), `mn_chunk_bytes` consecutive chunks along M/N (high word, stride offset).
+__device__ __forceinline__ uint32_t desc_lo_mn_major_plain(uint32_t saddr, uint32_t k_group_bytes) {
+    return ((saddr & 0x3FFFFu) >> 4) | (((k_group_bytes >> 4) & 0x3FFFu) << 16);
+}
+__host__ __device__ constexpr uint32_t desc_hi_plain(uint32_t mn_chunk_bytes) {
+    return ((mn_chunk_bytes >> 4) & 0x3FFFu) | (1u << 14);  // descriptor version 1, swizzle code 0
+}
 
 // Instruction descriptor for kind::f16 with bf16 A and B, fp32 D, M x N tile.
 // a_mn / b_mn: operand is MN-major (1) or K-major (0).
@@ -253,6 +269,21 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t 
         "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n"
         "}\n" ::"r"(d_tmem),
         "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
+        : "memory");
+}
+// The same with a separate high word for each operand (operands of different layouts).
+__device__ __forceinline__ void mma_ss_hi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                          uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        ".reg .b64 da, db;\n"
+        "mov.b64 da, {%1, %2};\n"
+        "mov.b64 db, {%3, %4};\n"
+        "setp.ne.b32 p, %6, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]; A holds bf16 pairs, one M row per lane, 16 K values per 8 columns.

@@ -269,7 +269,7 @@ def test_host_buffer_entry_point_equals_device_path(s2a, B, N, G, H, Hkv, d):
     dev = torch.device("cuda:0")
     qd, kd, vd, dOd = (x.to(dev) for x in (q, k, v, dO))
     o, lse = s2a.s2a_fwd(qd, kd, vd, G)
-    dq, dk, dv = s2a.s2a_bwd(qd, kd, vd, o, lse, dOd, G)
+    dq, dk, dv = s2a.s2a_bwd(qd, kd, vd, o, lse, dOd, G, fast=False)   # the host path below gets a minimum workspace too
     want = [x.cpu() for x in (o, lse, dq, dk, dv)]
     pin = [x.pin_memory() for x in (q, k, v, dO)]
     ws = torch.empty(max(s2a.bwd_workspace_bytes(B, N, H, Hkv, d, G), 256), dtype=torch.uint8, device=dev)
@@ -491,3 +491,40 @@ def test_benchmark_sizes_sampled_rows_and_properties(s2a, name, kv_tail):
         s = 0 if h < w.H // 2 else w.G // 2
         t_first = torch.tensor([(g * w.G + s) % w.N for g in range(w.N // w.G)], device=dev)
         assert torch.equal(o[0, t_first, h], vd[0, t_first, h // rep])
+
+
+@pytest.mark.parametrize("B,N,G,H,Hkv,d,kw,one_head_per_pass", [
+    (1, 1024, 256, 4, 4, 64, {}, False),
+    (2, 2048, 512, 8, 2, 128, {}, False),
+    (1, 2048, 512, 8, 2, 128, {}, True),                       # the KV heads in two passes
+    (1, 2400, 600, 4, 2, 128, {}, False),                      # ragged tiles
+    (1, 2400, 600, 4, 4, 64, {"leak_free": True}, True),
+    (1, 2400, 600, 4, 4, 128, {"swap_wrapped": True}, False),
+    (1, 4096, 1024, 6, 3, 128, {"n_unshifted": 2, "shift": 384}, False),
+    (1, 4096, 4096, 2, 2, 128, {"n_unshifted": 2}, False),     # full causal attention
+])
+def test_spilling_backward_equals_recomputing_backward(s2a, B, N, G, H, Hkv, d, kw, one_head_per_pass):
+    """With a workspace that has room for dS the dk/dv kernel spills it and dq is a plain product; with the
+    minimum workspace dq recomputes the scores.  dk and dv must agree bit for bit, dq to rounding, and dq
+    of the spilling path must match the oracle like any other result."""
+    q, k, v, dO = make_inputs(B, N, H, Hkv, d, seed=21)
+    dev = torch.device("cuda:0")
+    qd, kd, vd, dOd = (x.to(dev) for x in (q, k, v, dO))
+    o, lse = s2a.s2a_fwd_ex(qd, kd, vd, G, **kw)
+    mn = s2a.bwd_workspace_bytes(B, N, H, Hkv, d, G)
+    ref = s2a.s2a_bwd_ex(qd, kd, vd, o, lse, dOd, G, workspace=torch.empty(mn, dtype=torch.uint8, device=dev), **kw)
+    full = s2a.bwd_workspace_bytes_fast(B, N, H, Hkv, d, G, 1 << 40)
+    assert full > mn
+    # a shift that is not a multiple of 128 adds a tile per group: leave room for it
+    size = mn + 256 + (full - mn) // Hkv + 4096 if one_head_per_pass else full + (full - mn) // 2
+    got = tuple(torch.full_like(x, float("nan")) for x in (qd, kd, vd))
+    s2a.s2a_bwd_ex(qd, kd, vd, o, lse, dOd, G, workspace=torch.empty(size, dtype=torch.uint8, device=dev),
+                   dq=got[0], dk=got[1], dv=got[2], **kw)
+    torch.cuda.synchronize()
+    assert s2a.device_status() == (0, 0)
+    assert torch.equal(got[1], ref[1]) and torch.equal(got[2], ref[2])
+    assert not torch.isnan(got[0].float()).any()
+    assert rel_l2(got[0].double().cpu().numpy(), ref[0].double().cpu().numpy()) <= 2e-3
+    okw = dict(kw)
+    dq_ref, _, _ = orc.bwd(q, k, v, dO, G, **okw)
+    assert rel_l2(got[0].double().cpu().numpy(), dq_ref) <= GRAD_REL_L2

@@ -277,7 +277,14 @@ def run_ours(args):
     o = torch.empty_like(q)
     lse = torch.empty((B, H, N), dtype=torch.float32, device=dev)
     dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
-    ws = torch.empty(max(s2a.bwd_workspace_bytes(B, N, H, Hkv, d, G), 256), dtype=torch.uint8, device=dev)
+    # Backward workspace: with room for the spilled dS of every KV head (--bwd-workspace fast, the
+    # library's fastest path: dq is a plain product) or the minimum (dq recomputes the scores).
+    ws_min = s2a.bwd_workspace_bytes(B, N, H, Hkv, d, G)
+    ws_bytes = ws_min
+    if args.bwd_workspace == "fast":
+        ws_bytes = s2a.bwd_workspace_bytes_fast(B, N, H, Hkv, d, G, int(args.workspace_budget_gib * 2**30))
+    spilling = ws_bytes >= s2a.bwd_workspace_bytes_fast(B, N, H, Hkv, d, G, 1 << 50) > ws_min
+    ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 
     def step_plain():
@@ -376,7 +383,8 @@ def run_ours(args):
     peaks, peak_src = load_peaks()
     pairs = w.pairs
     alg_flops = {"fwd": 4 * d * pairs, "bwd_preprocess": 0, "bwd_dkdv": 8 * d * pairs, "bwd_dq": 2 * d * pairs}
-    exe_flops = {"fwd": 4 * d * pairs, "bwd_preprocess": 0, "bwd_dkdv": 8 * d * pairs, "bwd_dq": 6 * d * pairs}
+    exe_flops = {"fwd": 4 * d * pairs, "bwd_preprocess": 0, "bwd_dkdv": 8 * d * pairs,
+                 "bwd_dq": (2 if spilling else 6) * d * pairs}
     kernels = {}
     for n in names:
         ms = kernel_ms[n] / K
@@ -432,6 +440,8 @@ def run_ours(args):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "B": B, "N": N, "G": G, "H": H, "Hkv": Hkv, "d": d,
                    "l2": "inputs (5 x %.0f MB) larger than L2" % (q.numel() * 2 / 1e6),
+                   "bwd_workspace_bytes": ws_bytes,
+                   "bwd_dq": "product with spilled dS" if spilling else "recomputes S and dP",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "tokens_per_s": world * B * N * K / (total_ms_max * 1e-3),
         "clocks": clocks,
@@ -457,6 +467,9 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--bwd-workspace", choices=["fast", "min"], default="fast",
+                    help="backward workspace: room for the spilled dS of all KV heads (fast) or the minimum")
+    ap.add_argument("--workspace-budget-gib", type=float, default=24.0)
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -276,16 +276,22 @@ int s2a_fwd(const void* q, const void* k, const void* v, void* o, float* lse, in
     return s2a_fwd_ex(q, k, v, o, lse, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2, G / 2, 0u, stream);
 }
 
+namespace {
+// Workspace layout: D [B, H, N] fp32 padded to 256 bytes, 256 bytes of work counters for the persistent
+// kernels (together the minimum), then the spill area.
+constexpr size_t kCounterBytes = 256;
+size_t d_bytes(int B, int N, int H) {
+    return (static_cast<size_t>(B) * H * N * sizeof(float) + 255) & ~static_cast<size_t>(255);
+}
+}  // namespace
+
 size_t s2a_bwd_workspace_bytes(int B, int N, int H, int Hkv, int d, int G) {
     if (B <= 0 || N <= 0 || H <= 0 || Hkv <= 0 || d <= 0 || G <= 0) return 0;
     if (N % G != 0 || H % Hkv != 0) return 0;
-    const size_t bytes = static_cast<size_t>(B) * H * N * sizeof(float);
-    return (bytes + 255) & ~static_cast<size_t>(255);
+    return d_bytes(B, N, H) + kCounterBytes;
 }
 
 namespace {
-// Workspace layout: D [B, H, N] fp32 (the minimum), then 256 bytes of counters, then the spill area.
-constexpr size_t kSpillHeaderBytes = 256;
 constexpr size_t kSpillBlockBytes = static_cast<size_t>(kSpillBlockElems) * 2;
 // spill blocks of one KV head with its query heads, for groups of at most T tiles
 size_t spill_blocks_per_kv_head(int B, int N, int H, int Hkv, int G, int T) {
@@ -300,10 +306,10 @@ size_t s2a_bwd_workspace_bytes_fast(int B, int N, int H, int Hkv, int d, int G, 
     // otherwise one partial tile per run of the group that wraps
     const int T = (G % (2 * kTile) == 0) ? G / kTile : (G + kTile - 1) / kTile + 1;
     const size_t per_kv = spill_blocks_per_kv_head(B, N, H, Hkv, G, T) * kSpillBlockBytes;
-    if (budget <= min_bytes + kSpillHeaderBytes) return min_bytes;
-    size_t nk = (budget - min_bytes - kSpillHeaderBytes) / per_kv;
+    if (budget <= min_bytes) return min_bytes;
+    size_t nk = (budget - min_bytes) / per_kv;
     if (nk > static_cast<size_t>(Hkv)) nk = Hkv;
-    return nk == 0 ? min_bytes : min_bytes + kSpillHeaderBytes + nk * per_kv;
+    return nk == 0 ? min_bytes : min_bytes + nk * per_kv;
 }
 
 namespace {
@@ -364,11 +370,14 @@ int bwd_impl(const void* q, const void* k, const void* v, const void* o, const f
     const size_t min_bytes = s2a_bwd_workspace_bytes(B, N, H, Hkv, d, G);
     const size_t per_kv = spill_blocks_per_kv_head(B, N, H, Hkv, G, geo.tiles_per_group);
     size_t nk_fit = 0;
-    if (may_spill && workspace_bytes > min_bytes + kSpillHeaderBytes)
-        nk_fit = (workspace_bytes - min_bytes - kSpillHeaderBytes) / (per_kv * kSpillBlockBytes);
+    if (may_spill && workspace_bytes > min_bytes)
+        nk_fit = (workspace_bytes - min_bytes) / (per_kv * kSpillBlockBytes);
     if (nk_fit > static_cast<size_t>(Hkv)) nk_fit = Hkv;
     if (stages != kStageAll && nk_fit < static_cast<size_t>(Hkv)) nk_fit = 0;
 
+    char* base = static_cast<char*>(workspace);
+    int* counters = reinterpret_cast<int*>(base + d_bytes(B, N, H));  // [0] dK,dV kernel, [1] dQ-from-spill kernel
+    pk.counter = counters;
     cudaError_t e;
     if (stages & kStagePre) {
         e = launch_bwd_preprocess(pp, d, st);
@@ -376,7 +385,9 @@ int bwd_impl(const void* q, const void* k, const void* v, const void* o, const f
     }
     if (nk_fit == 0) {
         if (stages & kStageDkDv) {
-            e = launch_bwd_dkdv(pk, d, st);
+            e = cudaMemsetAsync(counters, 0, sizeof(int), st);
+            if (e != cudaSuccess) return cuda_fail(e);
+            e = launch_bwd_dkdv(pk, d, ds->n_sm, st);
             if (e != cudaSuccess) return cuda_fail(e);
         }
         if (stages & kStageDq) {
@@ -386,25 +397,25 @@ int bwd_impl(const void* q, const void* k, const void* v, const void* o, const f
         return S2A_OK;
     }
 
-    char* base = static_cast<char*>(workspace);
-    int* counter = reinterpret_cast<int*>(base + min_bytes);
-    pk.spill = reinterpret_cast<__nv_bfloat16*>(base + min_bytes + kSpillHeaderBytes);
+    pk.spill = reinterpret_cast<__nv_bfloat16*>(base + min_bytes);
     BwdDqSpillParams ps;
     memset(&ps, 0, sizeof ps);
     ps.tm_k = pq.tm_k;
     ps.spill = pk.spill;
-    ps.dq = pq.dq, ps.dq_tok_stride = pq.dq_tok_stride, ps.counter = counter;
+    ps.dq = pq.dq, ps.dq_tok_stride = pq.dq_tok_stride, ps.counter = counters + 1;
     ps.status = ds->status_ptr, ps.host_status = ds->host_word_dev, ps.geo = geo, ps.scale = scale;
     for (int hk0 = 0; hk0 < Hkv; hk0 += static_cast<int>(nk_fit)) {
         const int nk = Hkv - hk0 < static_cast<int>(nk_fit) ? Hkv - hk0 : static_cast<int>(nk_fit);
         pk.pass.hk0 = hk0, pk.pass.nk = nk;
         ps.pass = pk.pass;
         if (stages & kStageDkDv) {
-            e = launch_bwd_dkdv(pk, d, st);
+            e = cudaMemsetAsync(counters, 0, sizeof(int), st);
+            if (e != cudaSuccess) return cuda_fail(e);
+            e = launch_bwd_dkdv(pk, d, ds->n_sm, st);
             if (e != cudaSuccess) return cuda_fail(e);
         }
         if (stages & kStageDq) {
-            e = cudaMemsetAsync(counter, 0, sizeof(int), st);
+            e = cudaMemsetAsync(counters + 1, 0, sizeof(int), st);
             if (e != cudaSuccess) return cuda_fail(e);
             e = launch_bwd_dq_spill(ps, d, ds->n_sm, st);
             if (e != cudaSuccess) return cuda_fail(e);
@@ -583,7 +594,7 @@ namespace {
 // Built-in home for D = rowsum(dO * o) when the caller cannot provide a workspace: 2^20 fp32 rows
 // (4 MiB), which every GPU that loads this library keeps resident until the process exits.
 constexpr size_t kBuiltinScratchRows = size_t(1) << 20;
-static __device__ __align__(256) float g_builtin_scratch[kBuiltinScratchRows];
+static __device__ __align__(256) float g_builtin_scratch[kBuiltinScratchRows + kCounterBytes / sizeof(float)];
 
 // In host code `g_builtin_scratch` is only a handle for the runtime, not an address a kernel may
 // use; the device address is looked up once per device, with that device current.
@@ -620,7 +631,7 @@ int s2a_bwd_noalloc(const void* q, const void* k, const void* v, const void* o, 
     // Every row of D that the two gradient kernels read is rewritten by the first kernel of this
     // call, so nothing left in the array by an earlier call has to be cleared.
     return bwd_impl(q, k, v, o, lse, dO, dq, dk, dv, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2,
-                    G / 2, scratch, kBuiltinScratchRows * sizeof(float), stream, kStageAll, 0u, TokStrides(), false);
+                    G / 2, scratch, kBuiltinScratchRows * sizeof(float) + kCounterBytes, stream, kStageAll, 0u, TokStrides(), false);
 }
 
 size_t s2a_bwd_noalloc_max_rows(void) { return kBuiltinScratchRows; }

@@ -93,12 +93,6 @@ struct BwdCfg {
     static constexpr int kTmemCols = 512;
 };
 
-// Pack 32 fp32 values (as raw bits) into 16 bf16x2 words.
-__device__ __forceinline__ void pack32(const float (&x)[32], uint32_t (&out)[16]) {
-#pragma unroll
-    for (int e = 0; e < 16; ++e) out[e] = pack_bf16(x[2 * e], x[2 * e + 1]);
-}
-
 // Store COLS consecutive fp32 accumulator columns of this thread's tensor-memory lane (times `mul`)
 // as bf16 to `dst`.
 template <int COLS>
@@ -120,12 +114,6 @@ __device__ __forceinline__ void store_acc_cols(uint32_t t_addr, float mul, __nv_
         }
     }
 }
-
-// The elementwise warps come in two groups of four: group `half` handles columns [32*half, +32) of
-// each 64-column score buffer and writes its 32 bf16 results (16 packed columns) over the start of
-// its own columns, so the two groups never touch each other's columns.  The 64 K values of the
-// bf16 operand therefore sit at packed columns [0,16) and [32,48) of the buffer:
-__device__ __forceinline__ uint32_t packed_operand_col(int kk) { return (kk >> 1) * 32 + (kk & 1) * 8; }
 
 // Barrier block common to both kernels.
 template <int kStages>
@@ -480,8 +468,8 @@ __global__ void __launch_bounds__(DqCfg<HD>::kThreads, 1) s2a_bwd_dq_kernel(cons
 // ------------------------------------------------------------------------------------------------
 // 3. dK, dV
 // ------------------------------------------------------------------------------------------------
-// Tensor memory columns: dV [0,HD)  dK [128,128+HD)  S^T buffers [256,320) [320,384) [384,448)
-//                        dP^T [448,512)
+// Tensor memory columns: dV [0,HD)  dK [128,128+HD)  S^T buffers [256,320) [320,384)  dP^T [384,448)
+//                        K (bf16, the A operand of the score products) [448,448+HD/2)
 // One dP^T buffer is enough because the elementwise warps copy their part of it into registers at the
 // start of a step and release the buffer at once; that leaves room for a third S^T
 // buffer, and with three steps in flight the chain scores -> elementwise -> gradient MMAs of one
@@ -511,12 +499,74 @@ __device__ __forceinline__ HeadWalk head_walk(const Geometry& geo, int hq, int t
     return w;
 }
 
+// A work item of the dK,dV kernel: key tile `j0` (in the partition of the KV head's first query head) of
+// unit (b, hk, g0), in the block order shared by all kernels.  total_steps = 0 marks a slot of a group
+// that has fewer tiles than the largest one.
+struct DkDvItem {
+    int b, hk, tk0, k_valid, total_steps;
+};
+__device__ __forceinline__ DkDvItem dkdv_item(const Geometry& geo, const SpillPass& pass, long long id) {
+    DkDvItem t;
+    int unit, j0;
+    decode_block(id, geo.B * pass.nk * geo.groups, geo.tiles_per_group, &unit, &j0);
+    const int g0 = unit % geo.groups;
+    const int rep = geo.H / geo.Hkv;
+    t.hk = pass.hk0 + (unit / geo.groups) % pass.nk;
+    t.b = unit / (geo.groups * pass.nk);
+    const int hq0 = t.hk * rep;
+    const int s0 = (hq0 < geo.n_unshifted) ? 0 : geo.shift;
+    const GroupLayout L0 = group_layout(geo, s0, g0);
+    t.total_steps = 0;
+    t.tk0 = 0, t.k_valid = 0;
+    if (j0 >= L0.nTiles) return t;
+    const TileRef tk = tile_ref(L0, j0);
+    t.tk0 = tk.tok0;
+    t.k_valid = tk.valid;
+    for (int hq = hq0; hq < hq0 + rep; ++hq) {
+        const HeadWalk w = head_walk(geo, hq, t.tk0);
+        t.total_steps += w.n_end - w.n_begin;
+    }
+    return t;
+}
+
+// Barriers of the persistent dK,dV kernel.  Steps are counted through all items of the CTA (`it`), so
+// the rings of stages and score buffers simply carry on from one item to the next.
+template <int kStages>
+struct DkDvBars {
+    uint64_t res_full;            // K and V of an item landed (one phase per item)
+    uint64_t kt_full;             // K of an item has been copied into tensor memory
+    uint64_t kv_empty;            // the score products of an item are done: K and V may be overwritten
+    uint64_t acc_full;            // all gradient MMAs of an item are done
+    uint64_t acc_empty;           // the accumulators of an item have been read out
+    uint64_t drain;               // abort path only (gradient MMA warp)
+    uint64_t drain2;              // abort path only (score MMA warp)
+    uint64_t s_full[3];           // S^T of a step is in tensor memory (buffer it % 3)
+    uint64_t p_full[3];           // bf16 P^T and dS^T of a step are in tensor memory
+    uint64_t buf_free[3];         // gradient MMAs that read a score buffer's bf16 operands are done
+    uint64_t dp_free;             // the elementwise threads of a step hold their dP^T in registers
+    uint64_t st_full[kStages];    // streamed operands of a stage landed
+    uint64_t st_empty[kStages];   // MMAs reading a stage are done
+    uint64_t sched_full[8];       // a work item id has been published
+    long long item[8];
+    uint32_t tmem_slot;
+    int abort_flag;
+};
+
 // kSpill: every step's dS^T also goes to global memory (see SpillPass) for s2a_bwd_dq_spill_kernel.
+//
+// Persistent: one CTA per SM draws key tiles, heaviest first, from a counter in global memory.  The TMA
+// warp runs ahead across items (the K and V of the next item are fetched as soon as the last score
+// product of the current one has been issued and completed, its first query sub-tiles right behind),
+// so that barrier set-up, tensor-memory allocation, the first loads and the pipeline fill are paid
+// once per SM instead of once per key tile, and the score products of the next item run while the
+// accumulators of the finished one are written out.
 template <int HD, bool kSpill>
 __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(const __grid_constant__ BwdDkDvParams p) {
     using C = BwdCfg<HD>;
-    using Bars = BwdBars<C::kStages>;
-    constexpr int kBufs = 3;  // S^T buffers in flight
+    using Bars = DkDvBars<C::kStages>;
+    constexpr int kBufs = 2;   // S^T buffers in flight, one per elementwise group
+    constexpr int kSched = 8;  // item ids in flight: the TMA warp is at most five items ahead of the read-out
+    static_assert(C::kStages % 2 == 0, "a stage must always serve the same elementwise group");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sK = smem;                                // resident: K_j
@@ -524,6 +574,7 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
     uint8_t* sStage = sV + C::kBigTileBytes;           // per stage: Q_n then dO_n
     float* sStat = reinterpret_cast<float*>(sStage + C::kStages * C::kStageBytes);  // per stage: lse[64], D[64]
     Bars* bars = reinterpret_cast<Bars*>(reinterpret_cast<uint8_t*>(sStat) + C::kStages * 2 * C::kStatBytes);
+    static_assert(sizeof(Bars) <= C::kBarBytes, "barrier block");
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -536,43 +587,28 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
     if (s_poisoned != 0) return;
     const Geometry& geo = p.geo;
     const int rep = geo.H / geo.Hkv;
-
-    // key tile: enumerate in the rolled order of the first query head of the KV head, heaviest
-    // (earliest in the group) first
     const int Tg = geo.tiles_per_group;
-    int unit, j0;
-    decode_block(blockIdx.x, geo.B * p.pass.nk * geo.groups, Tg, &unit, &j0);
-    const int g0 = unit % geo.groups;
-    const int hk = p.pass.hk0 + (unit / geo.groups) % p.pass.nk;
-    const int b = unit / (geo.groups * p.pass.nk);
-    const int hq0 = hk * rep;
-    const int s0 = (hq0 < geo.n_unshifted) ? 0 : geo.shift;
-    const GroupLayout L0 = group_layout(geo, s0, g0);
-    if (j0 >= L0.nTiles) return;  // this group has fewer tiles than the largest one
-    const TileRef tk = tile_ref(L0, j0);
-    const int tk0 = tk.tok0;
-
-    int total_steps = 0;
-    for (int hq = hq0; hq < hq0 + rep; ++hq) {
-        const HeadWalk w = head_walk(geo, hq, tk0);
-        total_steps += w.n_end - w.n_begin;
-    }
+    const long long n_items = static_cast<long long>(geo.B) * p.pass.nk * geo.groups * Tg;
 
     if (threadIdx.x == 0) {
         mbar_init(&bars->res_full, 1);
+        mbar_init(&bars->kt_full, 256);
+        mbar_init(&bars->kv_empty, 1);
         mbar_init(&bars->acc_full, 1);
+        mbar_init(&bars->acc_empty, 256);
         mbar_init(&bars->drain, 1);
         mbar_init(&bars->drain2, 1);
         for (int x = 0; x < kBufs; ++x) {
             mbar_init(&bars->s_full[x], 1);
-            mbar_init(&bars->p_full[x], 256);
+            mbar_init(&bars->p_full[x], 128);   // the four elementwise warps whose turn the step is
             mbar_init(&bars->buf_free[x], 1);
         }
-        mbar_init(&bars->dp_free, 256);
+        mbar_init(&bars->dp_free, 128);
         for (int st = 0; st < C::kStages; ++st) {
             mbar_init(&bars->st_full[st], 1);
             mbar_init(&bars->st_empty[st], 1);
         }
+        for (int x = 0; x < kSched; ++x) mbar_init(&bars->sched_full[x], 1);
         bars->abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&p.tm_q);
@@ -589,44 +625,71 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_slot;
     const WaitCtx ctx{&bars->abort_flag, p.status, p.host_status};
-    constexpr uint32_t kColDV = 0, kColDK = 128, kColS = 256, kColP = 448;
+    constexpr uint32_t kColDV = 0, kColDK = 128, kColS = 256, kColP = 384, kColKt = 448;
+
+    // Every consumer role walks the same sequence of items: wait for the k-th id, stop at the end marker.
+    auto next_item = [&](int k, int where, long long* id) -> bool {
+        if (!mbar_wait(&bars->sched_full[k % kSched], (k / kSched) & 1, ctx, where)) return false;
+        *id = bars->item[k % kSched];
+        return *id < n_items;
+    };
 
     if (warp == 0) {
         if (lane == 0) {
-            mbar_expect_tx(&bars->res_full, 2 * C::kBigTileBytes);
-            for (int bx = 0; bx < C::kBoxes; ++bx) {
-                tma_load_4d(sK + bx * C::kBigBoxBytes, &p.tm_k, &bars->res_full, bx * 64, hk, tk0, b);
-                tma_load_4d(sV + bx * C::kBigBoxBytes, &p.tm_v, &bars->res_full, bx * 64, hk, tk0, b);
-            }
             int it = 0;
+            int last_res = -1;  // newest item whose K and V were requested
             bool ok = true;
-            for (int hq = hq0; ok && hq < hq0 + rep; ++hq) {
-                const HeadWalk w = head_walk(geo, hq, tk0);
-                for (int n = w.n_begin; n < w.n_end; ++n, ++it) {
-                    const int st = it % C::kStages;
-                    const uint32_t ph = (it / C::kStages) & 1;
-                    const TileRef tq = subtile_ref(w.L, n);
-                    const int tq0 = tq.tok0;
-                    // statistics of the valid rows only (a multiple of 4 rows, so of 16 bytes): a ragged
-                    // sub-tile must not read past the end of the arrays
-                    const uint32_t stat_bytes = static_cast<uint32_t>(tq.valid) * 4u;
-                    if (!mbar_wait(&bars->st_empty[st], ph ^ 1, ctx, kWaitBwdDkDv + 1)) { ok = false; break; }
-                    mbar_expect_tx(&bars->st_full[st], C::kStageBytes + 2 * stat_bytes);
-                    uint8_t* sQ = sStage + st * C::kStageBytes;
-                    uint8_t* sDO = sQ + C::kSubTileBytes;
-                    for (int bx = 0; bx < C::kBoxes; ++bx) {
-                        tma_load_4d(sQ + bx * C::kSubBoxBytes, &p.tm_q, &bars->st_full[st], bx * 64, hq, tq0, b);
-                        tma_load_4d(sDO + bx * C::kSubBoxBytes, &p.tm_do, &bars->st_full[st], bx * 64, hq, tq0, b);
-                    }
-                    const size_t stat_idx = (static_cast<size_t>(b) * geo.H + hq) * geo.N + tq0;
-                    if (stat_bytes != 0) {
-                        bulk_load_1d(sStat + st * 2 * kSubTile, p.lse + stat_idx, stat_bytes, &bars->st_full[st]);
-                        bulk_load_1d(sStat + st * 2 * kSubTile + kSubTile, p.Dsum + stat_idx, stat_bytes, &bars->st_full[st]);
+            for (int k = 0; ok; ++k) {
+                // draw the next item that has work; the other warps only see real items and the end marker
+                long long id;
+                DkDvItem t;
+                do {
+                    id = static_cast<long long>(atomicAdd(p.counter, 1));
+                    if (id >= n_items) break;
+                    t = dkdv_item(geo, p.pass, id);
+                } while (t.total_steps == 0);
+                bars->item[k % kSched] = id;
+                mbar_arrive(&bars->sched_full[k % kSched]);  // release: the id is visible to whoever sees the phase
+                if (id >= n_items) break;
+                // K and V of the item: their buffers are free once the score products of the previous item are done
+                if (k > 0 && !mbar_wait(&bars->kv_empty, (k - 1) & 1, ctx, kWaitBwdDkDv + 10)) break;
+                mbar_expect_tx(&bars->res_full, 2 * C::kBigTileBytes);
+                for (int bx = 0; bx < C::kBoxes; ++bx) {
+                    tma_load_4d(sK + bx * C::kBigBoxBytes, &p.tm_k, &bars->res_full, bx * 64, t.hk, t.tk0, t.b);
+                    tma_load_4d(sV + bx * C::kBigBoxBytes, &p.tm_v, &bars->res_full, bx * 64, t.hk, t.tk0, t.b);
+                }
+                last_res = k;
+                const int hq0 = t.hk * rep;
+                for (int hq = hq0; ok && hq < hq0 + rep; ++hq) {
+                    const HeadWalk w = head_walk(geo, hq, t.tk0);
+                    for (int n = w.n_begin; n < w.n_end; ++n, ++it) {
+                        const int st = it % C::kStages;
+                        const uint32_t ph = (it / C::kStages) & 1;
+                        const TileRef tq = subtile_ref(w.L, n);
+                        const int tq0 = tq.tok0;
+                        // statistics of the valid rows only (a multiple of 4 rows, so of 16 bytes): a ragged
+                        // sub-tile must not read past the end of the arrays
+                        const uint32_t stat_bytes = static_cast<uint32_t>(tq.valid) * 4u;
+                        if (!mbar_wait(&bars->st_empty[st], ph ^ 1, ctx, kWaitBwdDkDv + 1)) { ok = false; break; }
+                        mbar_expect_tx(&bars->st_full[st], C::kStageBytes + 2 * stat_bytes);
+                        uint8_t* sQ = sStage + st * C::kStageBytes;
+                        uint8_t* sDO = sQ + C::kSubTileBytes;
+                        for (int bx = 0; bx < C::kBoxes; ++bx) {
+                            tma_load_4d(sQ + bx * C::kSubBoxBytes, &p.tm_q, &bars->st_full[st], bx * 64, hq, tq0, t.b);
+                            tma_load_4d(sDO + bx * C::kSubBoxBytes, &p.tm_do, &bars->st_full[st], bx * 64, hq, tq0, t.b);
+                        }
+                        const size_t stat_idx = (static_cast<size_t>(t.b) * geo.H + hq) * geo.N + tq0;
+                        if (stat_bytes != 0) {
+                            bulk_load_1d(sStat + st * 2 * kSubTile, p.lse + stat_idx, stat_bytes, &bars->st_full[st]);
+                            bulk_load_1d(sStat + st * 2 * kSubTile + kSubTile, p.Dsum + stat_idx, stat_bytes, &bars->st_full[st]);
+                        }
                     }
                 }
             }
             if (bars->abort_flag != 0) {
-                mbar_wait_drain(&bars->res_full, 0);
+                // let loads that are still in flight land before the CTA gives its memory back: K and V of
+                // the newest item and the stages issued last
+                if (last_res >= 0) mbar_wait_drain(&bars->res_full, last_res & 1);
                 for (int nn = (it > C::kStages ? it - C::kStages : 0); nn < it; ++nn)
                     mbar_wait_drain(&bars->st_full[nn % C::kStages], (nn / C::kStages) & 1);
             }
@@ -637,35 +700,43 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         // elementwise warps hold the previous one in registers), then S^T = K Q^T into buffer it % 3
         // (warp-uniform loop, one elected lane issues; see the dQ kernel)
         constexpr uint32_t idesc_sc = idesc_bf16(128, kSubTile, 0, 0);
-        const uint32_t dK = desc_lo_k_major(smem_u32(sK)), dV = desc_lo_k_major(smem_u32(sV));
-        const uint32_t tP = tmem_base + kColP;
-        bool ok = mbar_wait_uniform(&bars->res_full, 0, ctx, kWaitBwdDkDv + 3);
-        for (int it = 0; ok && it < total_steps; ++it) {
-            const int st = it % C::kStages;
-            const int bf = it % kBufs;
-            if (!mbar_wait_uniform(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 2)) break;
-            if (it >= 1 && !mbar_wait_uniform(&bars->dp_free, (it - 1) & 1, ctx, kWaitBwdDkDv + 9)) break;
-            tc_fence_after();
-            const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
-            const uint32_t dQ = desc_lo_k_major(aQ), dDO = desc_lo_k_major(aQ + C::kSubTileBytes);
-            if (elect_one()) {
+        const uint32_t dV = desc_lo_k_major(smem_u32(sV));
+        const uint32_t tP = tmem_base + kColP, tKt = tmem_base + kColKt;
+        int it = 0;
+        bool ok = true;
+        for (int k = 0; ok; ++k) {
+            long long id = n_items;
+            if (!__all_sync(0xffffffffu, next_item(k, kWaitBwdDkDv + 11, &id) ? 1 : 0)) break;  // warp-uniform outcome
+            const DkDvItem t = dkdv_item(geo, p.pass, id);
+            if (!mbar_wait_uniform(&bars->res_full, k & 1, ctx, kWaitBwdDkDv + 3)) break;
+            if (!mbar_wait_uniform(&bars->kt_full, k & 1, ctx, kWaitBwdDkDv + 16)) break;
+            for (int x = 0; x < t.total_steps; ++x, ++it) {
+                const int st = it % C::kStages;
+                const int bf = it % kBufs;
+                if (!mbar_wait_uniform(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 2)) { ok = false; break; }
+                if (it >= 1 && !mbar_wait_uniform(&bars->dp_free, (it - 1) & 1, ctx, kWaitBwdDkDv + 9)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
+                const uint32_t dQ = desc_lo_k_major(aQ), dDO = desc_lo_k_major(aQ + C::kSubTileBytes);
+                if (elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk)
-                    mma_ss(tP, dV + desc_step_k_major(kk, C::kBigBoxBytes), dDO + desc_step_k_major(kk, C::kSubBoxBytes),
-                           idesc_sc, kk > 0);
-            }
-            __syncwarp();
-            if (it >= kBufs && !mbar_wait_uniform(&bars->buf_free[bf], ((it / kBufs) & 1) ^ 1, ctx, kWaitBwdDkDv + 8)) break;
-            tc_fence_after();
-            const uint32_t tS = tmem_base + kColS + bf * kSubTile;
-            if (elect_one()) {
+                    for (int kk = 0; kk < HD / 16; ++kk)
+                        mma_ss(tP, dV + desc_step_k_major(kk, C::kBigBoxBytes), dDO + desc_step_k_major(kk, C::kSubBoxBytes),
+                               idesc_sc, kk > 0);
+                }
+                __syncwarp();
+                if (it >= kBufs && !mbar_wait_uniform(&bars->buf_free[bf], ((it / kBufs) & 1) ^ 1, ctx, kWaitBwdDkDv + 8)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tS = tmem_base + kColS + bf * kSubTile;
+                if (elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk)
-                    mma_ss(tS, dK + desc_step_k_major(kk, C::kBigBoxBytes), dQ + desc_step_k_major(kk, C::kSubBoxBytes),
-                           idesc_sc, kk > 0);
-                mma_commit(&bars->s_full[bf]);
+                    for (int kk = 0; kk < HD / 16; ++kk)
+                        mma_ts(tS, tKt + 8 * kk, dQ + desc_step_k_major(kk, C::kSubBoxBytes), idesc_sc, kk > 0);
+                    mma_commit(&bars->s_full[bf]);
+                    if (x == t.total_steps - 1) mma_commit(&bars->kv_empty);  // nothing reads this item's K and V any more
+                }
+                __syncwarp();
             }
-            __syncwarp();
         }
         if (__any_sync(0xffffffffu, bars->abort_flag != 0)) {
             if (elect_one()) {
@@ -676,32 +747,39 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         __syncwarp();
     } else if (warp == 2) {
         // ---- gradient MMAs: dV += P^T dO and dK += dS^T Q of step `it`; both bf16 operands sit in
-        // the step's S^T buffer (P^T in the first 16 packed columns of each thread's 32, dS^T in the rest)
+        // the step's S^T buffer
         constexpr uint32_t idesc_acc = idesc_bf16(128, HD, 0, 1);
-        for (int it = 0; it < total_steps; ++it) {
-            const int st = it % C::kStages;
-            const int bf = it % kBufs;
-            if (!mbar_wait_uniform(&bars->p_full[bf], (it / kBufs) & 1, ctx, kWaitBwdDkDv + 4)) break;
-            tc_fence_after();
-            const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
-            const uint32_t dQmn = desc_lo_mn_major(aQ, C::kSubBoxBytes);
-            const uint32_t dDOmn = desc_lo_mn_major(aQ + C::kSubTileBytes, C::kSubBoxBytes);
-            const uint32_t tPt = tmem_base + kColS + bf * kSubTile;  // bf16 P^T
-            const uint32_t tdSt = tPt + 16;                          // bf16 dS^T
-            if (elect_one()) {
+        int it = 0;
+        bool ok = true;
+        for (int k = 0; ok; ++k) {
+            long long id = n_items;
+            if (!__all_sync(0xffffffffu, next_item(k, kWaitBwdDkDv + 12, &id) ? 1 : 0)) break;  // warp-uniform outcome
+            const DkDvItem t = dkdv_item(geo, p.pass, id);
+            for (int x = 0; x < t.total_steps; ++x, ++it) {
+                const int st = it % C::kStages;
+                const int bf = it % kBufs;
+                if (!mbar_wait_uniform(&bars->p_full[bf], (it / kBufs) & 1, ctx, kWaitBwdDkDv + 4)) { ok = false; break; }
+                // the first products of an item overwrite the accumulators: the previous item's must have been read out
+                if (x == 0 && k > 0 && !mbar_wait_uniform(&bars->acc_empty, (k - 1) & 1, ctx, kWaitBwdDkDv + 13)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t aQ = smem_u32(sStage + st * C::kStageBytes);
+                const uint32_t dQmn = desc_lo_mn_major(aQ, C::kSubBoxBytes);
+                const uint32_t dDOmn = desc_lo_mn_major(aQ + C::kSubTileBytes, C::kSubBoxBytes);
+                // the 16 queries of K slice kk: P^T in packed columns [16 kk, +8) of the buffer, dS^T in [16 kk + 8, +8)
+                const uint32_t tPt = tmem_base + kColS + bf * kSubTile;
+                if (elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < kSubTile / 16; ++kk)
-                    mma_ts(tmem_base + kColDV, tPt + packed_operand_col(kk), dDOmn + kk * kDescStepMn, idesc_acc,
-                           (it > 0) || (kk > 0));
+                    for (int kk = 0; kk < kSubTile / 16; ++kk)
+                        mma_ts(tmem_base + kColDV, tPt + 16 * kk, dDOmn + kk * kDescStepMn, idesc_acc, (x > 0) || (kk > 0));
 #pragma unroll
-                for (int kk = 0; kk < kSubTile / 16; ++kk)
-                    mma_ts(tmem_base + kColDK, tdSt + packed_operand_col(kk), dQmn + kk * kDescStepMn, idesc_acc,
-                           (it > 0) || (kk > 0));
-                mma_commit(&bars->st_empty[st]);
-                mma_commit(&bars->buf_free[bf]);
-                if (it == total_steps - 1) mma_commit(&bars->acc_full);
+                    for (int kk = 0; kk < kSubTile / 16; ++kk)
+                        mma_ts(tmem_base + kColDK, tPt + 16 * kk + 8, dQmn + kk * kDescStepMn, idesc_acc, (x > 0) || (kk > 0));
+                    mma_commit(&bars->st_empty[st]);
+                    mma_commit(&bars->buf_free[bf]);
+                    if (x == t.total_steps - 1) mma_commit(&bars->acc_full);
+                }
+                __syncwarp();
             }
-            __syncwarp();
         }
         if (__any_sync(0xffffffffu, bars->abort_flag != 0)) {
             if (elect_one()) {
@@ -713,132 +791,190 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
     } else if (warp == 3) {
         // spare warp: owns the tensor-memory allocation only
     } else {
+        // ---- elementwise.  The two groups of four warps take alternate steps: group (it & 1) handles step
+        // `it`, one thread per key row with all 64 query columns.  A step is a chain of long latencies
+        // (tensor-memory loads, exp2, tensor-memory stores, barrier round trips); alternating groups put
+        // one warp's waiting under the other's arithmetic.
         const int quad = warp & 3;
-        const int half = (warp - 4) >> 2;
+        const int group = (warp - 4) >> 2;
         const int row = quad * 32 + lane;  // key row of the tile owned by this thread
         const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
         const float c2 = p.scale_log2;
-        const bool key_valid = row < tk.valid;  // rows past the end of a ragged tile belong to other tiles
         bool ok = true;
         int it = 0;
-        for (int hq = hq0; ok && hq < hq0 + rep; ++hq) {
-            const HeadWalk w = head_walk(geo, hq, tk0);
-            // where this thread's 32 dS^T values of a step (four 16-byte chunks) go when they are spilled:
-            // chunks 4 half .. 4 half + 3 of key row `row` in block (j, n) of the spill unit (b, hq, g).  A
-            // block is stored chunk-major, so the 32 lanes of a warp write 512 contiguous bytes at a time.
-            uint4* spill_dst = nullptr;
-            if constexpr (kSpill) {
-                const long long su = (static_cast<long long>(b) * (p.pass.nk * rep) + (hq - p.pass.hk0 * rep)) * geo.groups + w.g;
-                spill_dst = reinterpret_cast<uint4*>(p.spill + spill_block(su, Tg, w.j, w.n_begin) * kSpillBlockElems) +
-                            half * 4 * kTile + row;
+        auto lds4 = [](uint32_t a) {
+            // explicit shared-memory loads: through a generic pointer they cost far more latency
+            float4 r;
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(a));
+            return r;
+        };
+        // K of item k goes from its shared-memory tile into tensor memory, where it is the A operand of
+        // S^T = K Q^T: an A operand in shared memory would be read again by every step (4 KB per MMA
+        // against 2 KB of B), and shared-memory bandwidth is what bounds this kernel.  Row `row`, columns
+        // [64 group, +64) of d: eight 16-byte chunks of the 128-byte-swizzled row, 32 packed columns.
+        auto copy_k = [&](int k) -> bool {
+            if (!mbar_wait(&bars->res_full, k & 1, ctx, kWaitBwdDkDv + 17)) return false;
+            if (group * 64 < HD) {
+                const uint32_t src = smem_u32(sK) + group * C::kBigBoxBytes + row * 128;
+                uint32_t kr[32];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(kr[4 * c]), "=r"(kr[4 * c + 1]), "=r"(kr[4 * c + 2]), "=r"(kr[4 * c + 3])
+                                 : "r"(src + ((c ^ (row & 7)) << 4)));
+                }
+                tmem_st_32x32(t_row + kColKt + group * 32, kr);
+                tmem_wait_st();
             }
-            for (int n = w.n_begin; n < w.n_end; ++n, ++it) {
-                const int st = it % C::kStages;
-                const int bf = it % kBufs;
-                // the statistics of this step travel with its stage
-                // s_full covers dP^T of this step as well: its MMAs were issued before those of S^T by the
-                // same thread, and a commit completes after everything issued before it
-                if (!mbar_wait(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 5) ||
-                    !mbar_wait(&bars->s_full[bf], (it / kBufs) & 1, ctx, kWaitBwdDkDv + 6)) {
-                    ok = false;
-                    break;
-                }
-                tc_fence_after();
-                // copy this thread's part of dP^T into registers and release the single dP^T buffer as
-                // soon as the copy has landed, so that the dP^T product of the next step runs while this
-                // step is worked on
-                uint32_t pr[32];
-                tmem_ld_32x32(t_row + kColP + half * 32, pr);
-                // lse[64] then D[64] of this stage; this thread's 32 columns start at float 32 * half.
-                // (explicit shared-memory loads: through a generic pointer they cost far more latency)
-                const uint32_t stat_sa = smem_u32(sStat + st * 2 * kSubTile) + half * 128;
-                auto lds4 = [](uint32_t a) {
-                    float4 r;
-                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(a));
-                    return r;
-                };
-                // this thread's 32 columns of S^T; its bf16 results go back over them once they are read:
-                // P^T into the first 16 (packed) columns, dS^T into the other 16
-                const uint32_t tS = t_row + kColS + bf * kSubTile + half * 32;
-                uint32_t sr[32];
-                tmem_ld_32x32(tS, sr);
-                tmem_wait_ld();
-                tc_fence_before();
-                mbar_arrive(&bars->dp_free);
-                uint32_t pkP[16], pkS[16];
-                // query x of this sub-tile sees key row r iff x is a valid row of the sub-tile and, in the
-                // diagonal tile, 128 j + r <= 64 n + x
-                const int q_valid = subtile_ref(w.L, n).valid;
-                if (n < w.n_begin + 2 || q_valid < kSubTile) {
-                    // masked sub-tiles: scalar path.  Statistics of rows that are not valid were never
-                    // loaded, so a masked entry is set to zero, never multiplied by zero.
-                    const int lim = (n < w.n_begin + 2) ? row - (n & 1) * kSubTile - half * 32 : -64;  // visible iff lim <= e < hi
-                    const int hi = q_valid - half * 32;
-                    float pt[32], ds[32];
-#pragma unroll
-                    for (int e4 = 0; e4 < 8; ++e4) {
-                        const float4 l = lds4(stat_sa + e4 * 16);
-                        const float4 dd = lds4(stat_sa + kSubTile * 4 + e4 * 16);
-                        const float lv[4] = {l.x, l.y, l.z, l.w};
-                        const float dv[4] = {dd.x, dd.y, dd.z, dd.w};
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int e = e4 * 4 + u;
-                            const bool visible = (e >= lim) && (e < hi);
-                            const float pe = fast_exp2(fmaf(__uint_as_float(sr[e]), c2, -lv[u] * kLog2e));
-                            pt[e] = visible ? pe : 0.f;
-                            ds[e] = visible ? pe * (__uint_as_float(pr[e]) - dv[u]) : 0.f;
-                        }
-                    }
-                    pack32(pt, pkP);
-                    pack32(ds, pkS);
-                } else {
-                    // two columns per instruction for the multiply-adds
-                    const uint64_t c2x2 = f2_pack(c2, c2), nl2e = f2_pack(-kLog2e, -kLog2e);
-#pragma unroll
-                    for (int e4 = 0; e4 < 8; ++e4) {
-                        const float4 l = lds4(stat_sa + e4 * 16);
-                        const float4 dd = lds4(stat_sa + kSubTile * 4 + e4 * 16);
-                        const uint64_t lp[2] = {f2_pack(l.x, l.y), f2_pack(l.z, l.w)};
-                        const uint64_t dp[2] = {f2_pack(dd.x, dd.y), f2_pack(dd.z, dd.w)};
-#pragma unroll
-                        for (int u = 0; u < 2; ++u) {
-                            const int e = e4 * 4 + 2 * u;
-                            const uint64_t x = f2_fma(f2_pack(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), c2x2,
-                                                      f2_mul(lp[u], nl2e));
-                            float x0, x1;
-                            f2_unpack(x, x0, x1);
-                            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-                            pkP[e >> 1] = pack_bf16(p0, p1);
-                            const uint64_t t = f2_sub(f2_pack(__uint_as_float(pr[e]), __uint_as_float(pr[e + 1])), dp[u]);
-                            float d0, d1;
-                            f2_unpack(f2_mul(f2_pack(p0, p1), t), d0, d1);
-                            pkS[e >> 1] = pack_bf16(d0, d1);
-                        }
-                    }
-                }
-                tmem_st_32x16(tS, pkP);
-                tmem_st_32x16(tS + 16, pkS);
+            tc_fence_before();
+            mbar_arrive(&bars->kt_full);
+            return true;
+        };
+        for (int k = 0; ok; ++k) {
+            long long id;
+            if (!next_item(k, kWaitBwdDkDv + 14, &id)) break;
+            if (k == 0 && !copy_k(0)) break;   // later items: copied at the end of the item before
+            const DkDvItem t = dkdv_item(geo, p.pass, id);
+            const bool key_valid = row < t.k_valid;  // rows past the end of a ragged tile belong to other tiles
+            const int hq0 = t.hk * rep;
+            for (int hq = hq0; ok && hq < hq0 + rep; ++hq) {
+                const HeadWalk w = head_walk(geo, hq, t.tk0);
+                // where this thread's dS^T values go when they are spilled: key row `row` of block (j, n) of the
+                // spill unit (b, hq, g).  A block is stored chunk-major (16-byte chunk c of row r at uint4 index
+                // c * 128 + r), so the 32 lanes of a warp write 512 contiguous bytes at a time.
+                uint4* spill_head = nullptr;
                 if constexpr (kSpill) {
-                    // streaming stores: written once, read once by the dQ kernel much later
+                    const long long su = (static_cast<long long>(t.b) * (p.pass.nk * rep) + (hq - p.pass.hk0 * rep)) * geo.groups + w.g;
+                    spill_head = reinterpret_cast<uint4*>(p.spill + spill_block(su, Tg, w.j, w.n_begin) * kSpillBlockElems) + row;
+                }
+                for (int n = w.n_begin; n < w.n_end; ++n, ++it) {
+                    if ((it & 1) != group) continue;
+                    const int st = it % C::kStages;
+                    const int bf = it % kBufs;
+                    // The statistics of this step travel with its stage (a stage always serves the same group:
+                    // kStages is even).  s_full covers dP^T of this step as well: its MMAs were issued before
+                    // those of S^T by the same thread, and a commit completes after everything issued before it.
+                    // A group sees only every other phase of s_full[bf]; the phase in between (step it - 3)
+                    // completed before S^T of step it - 2, which this group has waited for, so the parity test
+                    // cannot be fooled.
+                    if (!mbar_wait(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 5) ||
+                        !mbar_wait(&bars->s_full[bf], (it / kBufs) & 1, ctx, kWaitBwdDkDv + 6)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    // copy this thread's row of dP^T into registers and release the single dP^T buffer as soon as
+                    // the copy has landed, so that the dP^T product of the next step (the other group's) runs
+                    // while this step is worked on
+                    uint32_t pr[64];
+                    tmem_ld_32x32(t_row + kColP, *reinterpret_cast<uint32_t(*)[32]>(&pr[0]));
+                    tmem_ld_32x32(t_row + kColP + 32, *reinterpret_cast<uint32_t(*)[32]>(&pr[32]));
+                    // S^T comes 16 columns at a time, the next chunk in flight while the current one is worked on;
+                    // the bf16 results go back over the 16 columns just read: P^T into the first 8 (packed), dS^T
+                    // into the other 8
+                    const uint32_t tS = t_row + kColS + bf * kSubTile;
+                    uint32_t sbuf[2][16];
+                    tmem_ld_32x16(tS, sbuf[0]);
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    mbar_arrive(&bars->dp_free);
+                    const uint32_t stat_sa = smem_u32(sStat + st * 2 * kSubTile);  // lse[64] then D[64] of this stage
+                    // query x of this sub-tile sees key row r iff x is a valid row of the sub-tile and, in the
+                    // diagonal tile, 128 j + r <= 64 n + x
+                    const int q_valid = subtile_ref(w.L, n).valid;
+                    const bool masked = (n < w.n_begin + 2) || (q_valid < kSubTile);
+                    const int lim = (n < w.n_begin + 2) ? row - (n & 1) * kSubTile : -64;  // visible iff lim <= x < q_valid
+                    uint4* spill_dst = nullptr;
+                    if constexpr (kSpill) spill_dst = spill_head + static_cast<size_t>(n - w.n_begin) * (kSpillBlockElems / 8);
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        uint4 x = make_uint4(pkS[4 * c], pkS[4 * c + 1], pkS[4 * c + 2], pkS[4 * c + 3]);
-                        if (!key_valid) x = make_uint4(0u, 0u, 0u, 0u);
-                        __stcs(spill_dst + c * kTile, x);
+                        const uint32_t (&sr)[16] = sbuf[c & 1];
+                        if (c < 3) tmem_ld_32x16(tS + 16 * (c + 1), sbuf[(c + 1) & 1]);
+                        uint32_t pkP[8], pkS[8];
+                        if (masked) {
+                            // masked sub-tiles: scalar path.  Statistics of rows that are not valid were never
+                            // loaded, so a masked entry is set to zero, never multiplied by zero.
+#pragma unroll
+                            for (int e4 = 0; e4 < 4; ++e4) {
+                                const float4 l = lds4(stat_sa + (16 * c + 4 * e4) * 4);
+                                const float4 dd = lds4(stat_sa + kSubTile * 4 + (16 * c + 4 * e4) * 4);
+                                const float lv[4] = {l.x, l.y, l.z, l.w};
+                                const float dv[4] = {dd.x, dd.y, dd.z, dd.w};
+                                float pt[4], ds[4];
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    const int x = 16 * c + 4 * e4 + u;
+                                    const bool visible = (x >= lim) && (x < q_valid);
+                                    const float pe = fast_exp2(fmaf(__uint_as_float(sr[4 * e4 + u]), c2, -lv[u] * kLog2e));
+                                    pt[u] = visible ? pe : 0.f;
+                                    ds[u] = visible ? pe * (__uint_as_float(pr[x]) - dv[u]) : 0.f;
+                                }
+                                pkP[2 * e4] = pack_bf16(pt[0], pt[1]), pkP[2 * e4 + 1] = pack_bf16(pt[2], pt[3]);
+                                pkS[2 * e4] = pack_bf16(ds[0], ds[1]), pkS[2 * e4 + 1] = pack_bf16(ds[2], ds[3]);
+                            }
+                        } else {
+                            // two columns per instruction for the multiply-adds
+                            const uint64_t c2x2 = f2_pack(c2, c2), nl2e = f2_pack(-kLog2e, -kLog2e);
+#pragma unroll
+                            for (int e4 = 0; e4 < 4; ++e4) {
+                                const float4 l = lds4(stat_sa + (16 * c + 4 * e4) * 4);
+                                const float4 dd = lds4(stat_sa + kSubTile * 4 + (16 * c + 4 * e4) * 4);
+                                const uint64_t lp[2] = {f2_pack(l.x, l.y), f2_pack(l.z, l.w)};
+                                const uint64_t dp[2] = {f2_pack(dd.x, dd.y), f2_pack(dd.z, dd.w)};
+#pragma unroll
+                                for (int u = 0; u < 2; ++u) {
+                                    const int e = 4 * e4 + 2 * u;   // column within the chunk
+                                    const int x = 16 * c + e;       // query within the sub-tile
+                                    const uint64_t xs = f2_fma(f2_pack(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), c2x2,
+                                                               f2_mul(lp[u], nl2e));
+                                    float x0, x1;
+                                    f2_unpack(xs, x0, x1);
+                                    const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                                    pkP[e >> 1] = pack_bf16(p0, p1);
+                                    const uint64_t tt = f2_sub(f2_pack(__uint_as_float(pr[x]), __uint_as_float(pr[x + 1])), dp[u]);
+                                    float d0, d1;
+                                    f2_unpack(f2_mul(f2_pack(p0, p1), tt), d0, d1);
+                                    pkS[e >> 1] = pack_bf16(d0, d1);
+                                }
+                            }
+                        }
+                        tmem_st_32x8(tS + 16 * c, pkP);
+                        tmem_st_32x8(tS + 16 * c + 8, pkS);
+                        if constexpr (kSpill) {
+                            // streaming stores: written once, read once by the dQ kernel much later
+#pragma unroll
+                            for (int cc = 0; cc < 2; ++cc) {
+                                uint4 x = make_uint4(pkS[4 * cc], pkS[4 * cc + 1], pkS[4 * cc + 2], pkS[4 * cc + 3]);
+                                if (!key_valid) x = make_uint4(0u, 0u, 0u, 0u);
+                                __stcs(spill_dst + (2 * c + cc) * kTile, x);
+                            }
+                        }
+                        if (c < 3) tmem_wait_ld();
                     }
-                    spill_dst += kSpillBlockElems * 2 / sizeof(uint4);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(&bars->p_full[bf]);
                 }
-                tmem_wait_st();
-                tc_fence_before();
-                mbar_arrive(&bars->p_full[bf]);
             }
-        }
-        if (ok && mbar_wait(&bars->acc_full, 0, ctx, kWaitBwdDkDv + 7)) {
+            if (!ok) break;
+            // K of the next item, if there is one, while the last gradient MMAs of this one run: the TMA
+            // warp fetched it as soon as the last score product of this item was done (which also means that
+            // nothing reads the old copy any more)
+            {
+                long long next_id;
+                if (next_item(k + 1, kWaitBwdDkDv + 18, &next_id)) {
+                    if (!copy_k(k + 1)) break;
+                } else if (bars->abort_flag != 0) {
+                    break;
+                }
+            }
+            if (!mbar_wait(&bars->acc_full, k & 1, ctx, kWaitBwdDkDv + 7)) break;
             tc_fence_after();
-            const size_t out_row = (static_cast<size_t>(b) * geo.N + tk0 + row) * p.dkv_tok_stride + static_cast<size_t>(hk) * HD;
-            if (half == 0) store_acc_cols<HD>(t_row + kColDV, 1.0f, p.dv + out_row, key_valid);
+            const size_t out_row = (static_cast<size_t>(t.b) * geo.N + t.tk0 + row) * p.dkv_tok_stride + static_cast<size_t>(t.hk) * HD;
+            if (group == 0) store_acc_cols<HD>(t_row + kColDV, 1.0f, p.dv + out_row, key_valid);
             else store_acc_cols<HD>(t_row + kColDK, p.scale, p.dk + out_row, key_valid);
+            tc_fence_before();
+            mbar_arrive(&bars->acc_empty);
         }
     }
 
@@ -849,7 +985,6 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         tmem_dealloc(tmem_base, C::kTmemCols);
     }
 }
-
 
 // ------------------------------------------------------------------------------------------------
 // 4. dQ from spilled dS^T
@@ -1119,9 +1254,10 @@ cudaError_t launch_bwd_dq(const BwdDqParams& p, int d, cudaStream_t stream) {
     return cudaGetLastError();
 }
 
-cudaError_t launch_bwd_dkdv(const BwdDkDvParams& p, int d, cudaStream_t stream) {
+cudaError_t launch_bwd_dkdv(const BwdDkDvParams& p, int d, int n_sm, cudaStream_t stream) {
     const Geometry& g = p.geo;
-    const unsigned grid = static_cast<unsigned>(static_cast<long long>(g.B) * p.pass.nk * g.groups * g.tiles_per_group);
+    const long long items = static_cast<long long>(g.B) * p.pass.nk * g.groups * g.tiles_per_group;
+    const unsigned grid = static_cast<unsigned>(items < n_sm ? items : n_sm);
     if (p.spill != nullptr) {
         if (d == 64) s2a_bwd_dkdv_kernel<64, true><<<grid, BwdCfg<64>::kThreads, BwdCfg<64>::kSmemBytes, stream>>>(p);
         else s2a_bwd_dkdv_kernel<128, true><<<grid, BwdCfg<128>::kThreads, BwdCfg<128>::kSmemBytes, stream>>>(p);

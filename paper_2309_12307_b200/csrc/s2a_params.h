@@ -169,6 +169,7 @@ struct alignas(64) BwdDkDvParams {
     long long dkv_tok_stride;  // elements between consecutive tokens of dk and dv (Hkv * d when dense)
     __nv_bfloat16* spill;      // dS^T blocks of this pass (spilling variant only)
     SpillPass pass;            // KV heads this launch covers (all of them when nothing is spilled)
+    int* counter;              // next work item; zero when the kernel starts
     int* status;       // device status word (see WaitCtx)
     int* host_status;  // its mirror in mapped host memory
     Geometry geo;
@@ -193,7 +194,7 @@ struct alignas(64) BwdDqSpillParams {
 cudaError_t launch_fwd(const FwdParams& p, int d, cudaStream_t stream);
 cudaError_t launch_bwd_preprocess(const PreParams& p, int d, cudaStream_t stream);
 cudaError_t launch_bwd_dq(const BwdDqParams& p, int d, cudaStream_t stream);
-cudaError_t launch_bwd_dkdv(const BwdDkDvParams& p, int d, cudaStream_t stream);  // p.spill != nullptr: spilling variant
+cudaError_t launch_bwd_dkdv(const BwdDkDvParams& p, int d, int n_sm, cudaStream_t stream);  // persistent; p.spill != nullptr: spilling variant
 cudaError_t launch_bwd_dq_spill(const BwdDqSpillParams& p, int d, int n_sm, cudaStream_t stream);  // persistent: one CTA per SM
 
 // Per-device kernel attribute set-up (dynamic shared memory sizes).

@@ -55,8 +55,9 @@ def test_version_and_status_strings(lib):
 def test_workspace_bytes(lib):
     lib.s2a_bwd_workspace_bytes.restype = ctypes.c_size_t
     f = lib.s2a_bwd_workspace_bytes
-    assert f(1, 32768, 32, 32, 128, 8192) == 1 * 32 * 32768 * 4
-    assert f(1, 1024, 4, 4, 64, 256) == 4 * 1024 * 4
+    # D [B, H, N] in fp32, padded to 256 bytes, and 256 bytes of work counters
+    assert f(1, 32768, 32, 32, 128, 8192) == 1 * 32 * 32768 * 4 + 256
+    assert f(1, 1024, 4, 4, 64, 256) == 4 * 1024 * 4 + 256
     assert f(1, 1000, 4, 4, 64, 256) == 0      # N % G
     assert f(1, 1024, 6, 4, 64, 256) == 0      # H % Hkv
     assert f(0, 1024, 4, 4, 64, 256) == 0
@@ -89,3 +90,21 @@ def test_bad_arguments_are_rejected_without_a_device(lib):
     lib.s2a_bwd.argtypes = [P] * 9 + [ctypes.c_int] * 6 + [P, ctypes.c_size_t, P]
     assert lib.s2a_bwd(a, a, a, a, a, a, a, a, a, 1, 1024, 4, 4, 64, 256, a, 16, None) == -1
     assert lib.s2a_bwd(a, a, a, a, a, a, a, a, a, 1, 1024, 4, 4, 64, 256, None, 1 << 20, None) == -1
+
+
+def test_fast_workspace_bytes(lib):
+    lib.s2a_bwd_workspace_bytes.restype = ctypes.c_size_t
+    lib.s2a_bwd_workspace_bytes_fast.restype = ctypes.c_size_t
+    lib.s2a_bwd_workspace_bytes_fast.argtypes = [ctypes.c_int] * 6 + [ctypes.c_size_t]
+    f, g = lib.s2a_bwd_workspace_bytes, lib.s2a_bwd_workspace_bytes_fast
+    mn = f(1, 32768, 32, 32, 128, 8192)
+    blocks_per_unit = 64 * 65                      # T (T + 1) with T = 8192 / 128 tiles per group
+    per_kv = 1 * 1 * 4 * blocks_per_unit * 16384   # B * (H / Hkv) * (N / G) units of 16 KiB blocks
+    assert g(1, 32768, 32, 32, 128, 8192, 1 << 40) == mn + 32 * per_kv
+    assert g(1, 32768, 32, 32, 128, 8192, mn + 3 * per_kv + 5) == mn + 3 * per_kv      # whole KV heads only
+    assert g(1, 32768, 32, 32, 128, 8192, mn + per_kv - 1) == mn                       # not even one fits
+    assert g(1, 32768, 32, 32, 128, 8192, 0) == mn
+    assert g(1, 1000, 4, 4, 64, 256, 1 << 40) == 0                                     # invalid sizes
+    # ragged groups (G / 2 not a multiple of 128): one more tile per run of the wrapped group
+    T = (25000 + 127) // 128 + 1
+    assert g(1, 100000, 32, 32, 128, 25000, 1 << 50) == f(1, 100000, 32, 32, 128, 25000) + 32 * 4 * T * (T + 1) * 16384

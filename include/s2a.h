@@ -216,13 +216,15 @@ int s2a_bwd_stage(const void* q, const void* k, const void* v, const void* o, co
 /*
  * Forward + backward from HOST buffers (pinned memory, or the copies are not asynchronous): q, k, v,
  * dO go to the caller's device buffers, s2a_fwd and s2a_bwd run there, and o, lse, dq, dk, dv come
- * back.  Heads are independent, so the work is cut into up to 16 chunks of whole KV heads - one KV head
+ * back.  Heads are independent, so the work is cut into up to 16 chunks of whole KV heads - small ones
  * at either end, growing towards the middle - and the copy of one chunk, the kernels of the previous
  * one and the copy back of the one before that overlap (two copy streams owned by the library,
  * created by the first call on a device, ordered
  * against `stream` by events).  Everything is ordered after the work already in `stream` and
  * `stream` is complete only when the last result has landed: the caller synchronises `stream`
- * before reading the host outputs.  Results are bit-identical to s2a_fwd + s2a_bwd.
+ * before reading the host outputs.  Results are bit-identical to s2a_fwd + s2a_bwd given the same
+ * workspace size (which selects how dq is computed, see s2a_bwd; what counts here is how many KV heads
+ * of the largest chunk the workspace has dS room for).
  *   h_*  : host pointers, same layouts and types as the device tensors
  *   d_*  : device buffers of the same sizes, owned by the caller (the library allocates no memory);
  *          used as staging space: their contents after the call are unspecified

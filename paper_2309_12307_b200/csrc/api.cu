@@ -492,8 +492,10 @@ int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const vo
     // Heads are independent, so the job is cut into chunks of whole KV heads (with their query heads):
     // while chunk c is computed, chunk c+1 travels to the device and the results of chunk c-1 travel
     // back.  Only the first chunk's upload and the last chunk's download cannot be hidden, so the
-    // chunks at both ends are small (one KV head) and grow towards the middle, where wide rows keep
-    // the strided copies efficient: 1,1,2,4,8,8,4,2,1,1 KV heads for Hkv = 32.  Chunk c holds the KV
+    // chunks at both ends are small and grow towards the middle, where wide rows keep the strided
+    // copies efficient: 2,2,4,8,8,4,2,2 KV heads for Hkv = 32 (a chunk of a single 256-byte head row per
+    // token copies at well under the link's rate, which costs more than its shorter exposure saves).
+    // Chunk c holds the KV
     // heads [kv0[c], kv0[c] + kvn[c]) and sits densely ([B, N, heads of the chunk, d]) at the matching
     // offset of the caller's device buffers.
     const int rep = H / Hkv;
@@ -501,13 +503,14 @@ int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const vo
     int chunks = 0;
     {
         int left[kMaxHostChunks / 2], right[kMaxHostChunks / 2], nl = 0, nr = 0;
-        int remaining = Hkv, size = 1, uses = 0;
+        const int first = Hkv >= 32 ? Hkv / 16 : 1;
+        int remaining = Hkv, size = first, uses = 0;
         const int cap = Hkv >= 8 ? Hkv / 4 : 1;
         while (remaining > 0) {
             const int a = size < remaining ? size : remaining;
             if (nl <= nr) left[nl++] = a; else right[nr++] = a;
             remaining -= a;
-            if (++uses == (size == 1 ? 4 : 2)) {   // 1,1 at each end, then every size once per end
+            if (++uses == (size == first ? 4 : 2)) {   // the smallest size twice at each end, then every size once per end
                 uses = 0;
                 if (size * 2 <= cap) size *= 2;
             }

@@ -31,10 +31,26 @@ UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "llama2_7b_32k"
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 # DRAM bytes (read + write) per launch, from one ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum) of each kernel on llama2_7b_8k; every tensor is touched once, so traffic
-# scales with B*N*(H+Hkv)*d.  An entry is None once its kernel has changed since the capture.
-NCU_TRAFFIC_8K = {"fwd": 249.6e6, "bwd_preprocess": 137.9e6, "bwd_dkdv": 375.1e6, "bwd_dq": 322.8e6}
+# dram__bytes_write.sum) of each kernel on llama2_7b_8k.  The tensors q, k, v, o, dO, dq, dk, dv are
+# each touched once, so that part scales with B*N*(H+Hkv)*d; the spilled dS (written by the dK/dV
+# kernel, read by the dQ product kernel) is 2 bytes per entry of every 128 x 64 block and scales with
+# the number of blocks.  An entry is None where the kernel has changed since its capture.
+#   name: (bytes that scale with the tensors, bytes that scale with the spill) at 8k
+NCU_TRAFFIC_8K = {
+    "fwd": (249.6e6, 0.0),
+    "bwd_preprocess": (137.9e6, 0.0),
+    "bwd_dkdv": None,                               # recomputing backward: persistent form not captured
+    "bwd_dq": (322.8e6, 0.0),
+    "bwd_dkdv_spill": (919.9e6 - 570.4e6, 570.4e6),  # 271.0 MB read + 648.9 MB written, 570.4 MB of it the spill
+    "bwd_dq_spill": (696.6e6 - 570.4e6, 570.4e6),    # 637.7 MB read + 58.9 MB written
+}
 NCU_TRAFFIC_8K_SIZE = 1 * 8192 * (32 + 32) * 128
+NCU_SPILL_8K_BLOCKS = 32 * 4 * 16 * 17             # units x T (T + 1) blocks of 16 KiB, T = 2048 / 128
+
+
+def spill_blocks(w):
+    T = w.G // 128 if w.G % 256 == 0 else (w.G + 127) // 128 + 1
+    return w.B * w.H * (w.N // w.G) * T * (T + 1)
 
 
 def load_peaks():
@@ -403,9 +419,10 @@ def run_ours(args):
         regime = "sustained" if capped else "burst"
     peak = peak_sustained if regime == "sustained" else peak_burst
     achieved = kernels[dom]["algorithmic_tflops"]
-    traffic = NCU_TRAFFIC_8K.get(dom)
+    traffic = NCU_TRAFFIC_8K.get(dom + "_spill" if spilling and dom in ("bwd_dkdv", "bwd_dq") else dom)
     if traffic is not None:
-        traffic = traffic * (B * N * (H + Hkv) * d) / NCU_TRAFFIC_8K_SIZE
+        traffic = (traffic[0] * (B * N * (H + Hkv) * d) / NCU_TRAFFIC_8K_SIZE
+                   + traffic[1] * spill_blocks(w) / NCU_SPILL_8K_BLOCKS)
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": traffic, "traffic_unit": "bytes per launch (ncu on 8k, scaled)",
                 "peak_source": f"{peak_src} bf16 {regime} (chosen from this run's clock record)",

@@ -177,9 +177,9 @@ int s2a_bwd_packed(const void* qkv, const void* o, const float* lse, const void*
  * initialisation.  s2a_bwd wants a workspace from such a caller; this variant does not.
  *
  * It computes exactly what s2a_bwd computes with a minimum workspace (same kernels, same results), but keeps
- * D = rowsum(dO * o) in an array that is part of the library image: 2^20 fp32 values (4 MiB) on
- * every GPU that loads the library, held until the process exits.  It calls no allocation routine
- * of any kind.
+ * D = rowsum(dO * o) and the work counter of its persistent kernel in an array that is part of the
+ * library image: 2^20 fp32 values and 256 bytes (4 MiB in all) on every GPU that loads the library,
+ * held until the process exits.  It calls no allocation routine of any kind.
  *
  *   Limit     : B * H * N <= s2a_bwd_noalloc_max_rows() (= 1,048,576; e.g. B=1, H=32, N=32768).
  *               Larger problems return S2A_ERR_TOO_LARGE and enqueue nothing; use s2a_bwd.
@@ -189,8 +189,9 @@ int s2a_bwd_packed(const void* qkv, const void* o, const float* lse, const void*
  *               and safe.  Two calls that can run on the GPU at the same time (different streams,
  *               or different host threads on different streams) overwrite each other's D and
  *               give wrong gradients: serialise them, or use s2a_bwd with separate workspaces.
- *   Contents  : the array keeps whatever the previous call left; every value a call reads is
- *               first rewritten by that same call, so nothing needs clearing in between.
+ *   Contents  : the array keeps whatever the previous call left; every value of D a call reads is
+ *               first rewritten by that same call, and the work counter is set to zero by a 4-byte
+ *               memset on `stream` ahead of the kernel that counts with it, so the caller clears nothing.
  * Other arguments, shapes, errors and the meaning of `stream` are those of s2a_bwd.
  */
 int s2a_bwd_noalloc(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* dO,

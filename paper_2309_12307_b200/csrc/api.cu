@@ -594,8 +594,9 @@ int s2a_fwd_bwd_host(const void* h_q, const void* h_k, const void* h_v, const vo
 // ---------------------------------------------------------------------------------------------
 namespace {
 
-// Built-in home for D = rowsum(dO * o) when the caller cannot provide a workspace: 2^20 fp32 rows
-// (4 MiB), which every GPU that loads this library keeps resident until the process exits.
+// Built-in home for D = rowsum(dO * o) and the work counters when the caller cannot provide a
+// workspace: 2^20 fp32 rows and 256 bytes (4 MiB in all), which every GPU that loads this library keeps
+// resident until the process exits.
 constexpr size_t kBuiltinScratchRows = size_t(1) << 20;
 static __device__ __align__(256) float g_builtin_scratch[kBuiltinScratchRows + kCounterBytes / sizeof(float)];
 
@@ -632,7 +633,8 @@ int s2a_bwd_noalloc(const void* q, const void* k, const void* v, const void* o, 
     const int rc = builtin_scratch(&scratch);
     if (rc != S2A_OK) return rc;
     // Every row of D that the two gradient kernels read is rewritten by the first kernel of this
-    // call, so nothing left in the array by an earlier call has to be cleared.
+    // call and the work counter is cleared by a memset ahead of its kernel, so nothing left in the
+    // array by an earlier call matters.
     return bwd_impl(q, k, v, o, lse, dO, dq, dk, dv, B, N, H, Hkv, d, G, 1.0f / sqrtf(static_cast<float>(d)), H / 2,
                     G / 2, scratch, kBuiltinScratchRows * sizeof(float) + kCounterBytes, stream, kStageAll, 0u, TokStrides(), false);
 }

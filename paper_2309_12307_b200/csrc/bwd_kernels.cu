@@ -564,9 +564,10 @@ template <int HD, bool kSpill>
 __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(const __grid_constant__ BwdDkDvParams p) {
     using C = BwdCfg<HD>;
     using Bars = DkDvBars<C::kStages>;
-    constexpr int kBufs = 2;   // S^T buffers in flight, one per elementwise group
+    constexpr int kBufs = 2;   // S^T buffers in flight
+    constexpr int kCols = 32;  // query columns per elementwise thread and step: two threads share a key row
+    constexpr int kChunks = kCols / 16;
     constexpr int kSched = 8;  // item ids in flight: the TMA warp is at most five items ahead of the read-out
-    static_assert(C::kStages % 2 == 0, "a stage must always serve the same elementwise group");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sK = smem;                                // resident: K_j
@@ -600,10 +601,10 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
         mbar_init(&bars->drain2, 1);
         for (int x = 0; x < kBufs; ++x) {
             mbar_init(&bars->s_full[x], 1);
-            mbar_init(&bars->p_full[x], 128);   // the four elementwise warps whose turn the step is
+            mbar_init(&bars->p_full[x], 256);
             mbar_init(&bars->buf_free[x], 1);
         }
-        mbar_init(&bars->dp_free, 128);
+        mbar_init(&bars->dp_free, 256);
         for (int st = 0; st < C::kStages; ++st) {
             mbar_init(&bars->st_full[st], 1);
             mbar_init(&bars->st_empty[st], 1);
@@ -791,10 +792,11 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
     } else if (warp == 3) {
         // spare warp: owns the tensor-memory allocation only
     } else {
-        // ---- elementwise.  The two groups of four warps take alternate steps: group (it & 1) handles step
-        // `it`, one thread per key row with all 64 query columns.  A step is a chain of long latencies
-        // (tensor-memory loads, exp2, tensor-memory stores, barrier round trips); alternating groups put
-        // one warp's waiting under the other's arithmetic.
+        // ---- elementwise.  Thread (quad, lane, group) owns key row 32 quad + lane and the query columns
+        // [32 group, +32) of every step.  (Letting the two groups of four warps take alternate steps with a
+        // whole row per thread was measured too: with two S^T buffers the chain S^T -> elementwise ->
+        // gradient MMAs of a buffer is what a step waits for, and half the columns per thread halve its
+        // elementwise part: 3.33 against 3.53 ms on the Llama2-7B 32k shape.)
         const int quad = warp & 3;
         const int group = (warp - 4) >> 2;
         const int row = quad * 32 + lane;  // key row of the tile owned by this thread
@@ -848,33 +850,29 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                     spill_head = reinterpret_cast<uint4*>(p.spill + spill_block(su, Tg, w.j, w.n_begin) * kSpillBlockElems) + row;
                 }
                 for (int n = w.n_begin; n < w.n_end; ++n, ++it) {
-                    if ((it & 1) != group) continue;
+                    const int cg0 = 2 * group;   // first 16-column chunk of this thread
                     const int st = it % C::kStages;
                     const int bf = it % kBufs;
-                    // The statistics of this step travel with its stage (a stage always serves the same group:
-                    // kStages is even).  s_full covers dP^T of this step as well: its MMAs were issued before
-                    // those of S^T by the same thread, and a commit completes after everything issued before it.
-                    // A group sees only every other phase of s_full[bf]; the phase in between (step it - 3)
-                    // completed before S^T of step it - 2, which this group has waited for, so the parity test
-                    // cannot be fooled.
+                    // The statistics of this step travel with its stage.  s_full covers dP^T of this step as
+                    // well: its MMAs were issued before those of S^T by the same thread, and a commit completes
+                    // after everything issued before it.
                     if (!mbar_wait(&bars->st_full[st], (it / C::kStages) & 1, ctx, kWaitBwdDkDv + 5) ||
                         !mbar_wait(&bars->s_full[bf], (it / kBufs) & 1, ctx, kWaitBwdDkDv + 6)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    // copy this thread's row of dP^T into registers and release the single dP^T buffer as soon as
-                    // the copy has landed, so that the dP^T product of the next step (the other group's) runs
-                    // while this step is worked on
-                    uint32_t pr[64];
-                    tmem_ld_32x32(t_row + kColP, *reinterpret_cast<uint32_t(*)[32]>(&pr[0]));
-                    tmem_ld_32x32(t_row + kColP + 32, *reinterpret_cast<uint32_t(*)[32]>(&pr[32]));
-                    // S^T comes 16 columns at a time, the next chunk in flight while the current one is worked on;
-                    // the bf16 results go back over the 16 columns just read: P^T into the first 8 (packed), dS^T
-                    // into the other 8
+                    // copy this thread's part of dP^T into registers and release the single dP^T buffer as soon
+                    // as the copy has landed, so that the dP^T product of the next step runs while this step is
+                    // worked on
+                    uint32_t pr[kCols];
+                    tmem_ld_32x32(t_row + kColP + 16 * cg0, pr);
+                    // S^T in two chunks of 16 columns; the bf16 results of a chunk go back over its 16 columns:
+                    // P^T into the first 8 (packed), dS^T into the other 8
                     const uint32_t tS = t_row + kColS + bf * kSubTile;
                     uint32_t sbuf[2][16];
-                    tmem_ld_32x16(tS, sbuf[0]);
+                    tmem_ld_32x16(tS + 16 * cg0, sbuf[0]);
+                    tmem_ld_32x16(tS + 16 * (cg0 + 1), sbuf[1]);
                     tmem_wait_ld();
                     tc_fence_before();
                     mbar_arrive(&bars->dp_free);
@@ -887,27 +885,27 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                     uint4* spill_dst = nullptr;
                     if constexpr (kSpill) spill_dst = spill_head + static_cast<size_t>(n - w.n_begin) * (kSpillBlockElems / 8);
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const uint32_t (&sr)[16] = sbuf[c & 1];
-                        if (c < 3) tmem_ld_32x16(tS + 16 * (c + 1), sbuf[(c + 1) & 1]);
+                    for (int c = 0; c < kChunks; ++c) {
+                        const int cg = cg0 + c;   // chunk within the sub-tile: queries [16 cg, +16)
+                        const uint32_t (&sr)[16] = sbuf[c];
                         uint32_t pkP[8], pkS[8];
                         if (masked) {
                             // masked sub-tiles: scalar path.  Statistics of rows that are not valid were never
                             // loaded, so a masked entry is set to zero, never multiplied by zero.
 #pragma unroll
                             for (int e4 = 0; e4 < 4; ++e4) {
-                                const float4 l = lds4(stat_sa + (16 * c + 4 * e4) * 4);
-                                const float4 dd = lds4(stat_sa + kSubTile * 4 + (16 * c + 4 * e4) * 4);
+                                const float4 l = lds4(stat_sa + (16 * cg + 4 * e4) * 4);
+                                const float4 dd = lds4(stat_sa + kSubTile * 4 + (16 * cg + 4 * e4) * 4);
                                 const float lv[4] = {l.x, l.y, l.z, l.w};
                                 const float dv[4] = {dd.x, dd.y, dd.z, dd.w};
                                 float pt[4], ds[4];
 #pragma unroll
                                 for (int u = 0; u < 4; ++u) {
-                                    const int x = 16 * c + 4 * e4 + u;
+                                    const int x = 16 * cg + 4 * e4 + u;   // query within the sub-tile
                                     const bool visible = (x >= lim) && (x < q_valid);
                                     const float pe = fast_exp2(fmaf(__uint_as_float(sr[4 * e4 + u]), c2, -lv[u] * kLog2e));
                                     pt[u] = visible ? pe : 0.f;
-                                    ds[u] = visible ? pe * (__uint_as_float(pr[x]) - dv[u]) : 0.f;
+                                    ds[u] = visible ? pe * (__uint_as_float(pr[16 * c + 4 * e4 + u]) - dv[u]) : 0.f;
                                 }
                                 pkP[2 * e4] = pack_bf16(pt[0], pt[1]), pkP[2 * e4 + 1] = pack_bf16(pt[2], pt[3]);
                                 pkS[2 * e4] = pack_bf16(ds[0], ds[1]), pkS[2 * e4 + 1] = pack_bf16(ds[2], ds[3]);
@@ -917,14 +915,14 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                             const uint64_t c2x2 = f2_pack(c2, c2), nl2e = f2_pack(-kLog2e, -kLog2e);
 #pragma unroll
                             for (int e4 = 0; e4 < 4; ++e4) {
-                                const float4 l = lds4(stat_sa + (16 * c + 4 * e4) * 4);
-                                const float4 dd = lds4(stat_sa + kSubTile * 4 + (16 * c + 4 * e4) * 4);
+                                const float4 l = lds4(stat_sa + (16 * cg + 4 * e4) * 4);
+                                const float4 dd = lds4(stat_sa + kSubTile * 4 + (16 * cg + 4 * e4) * 4);
                                 const uint64_t lp[2] = {f2_pack(l.x, l.y), f2_pack(l.z, l.w)};
                                 const uint64_t dp[2] = {f2_pack(dd.x, dd.y), f2_pack(dd.z, dd.w)};
 #pragma unroll
                                 for (int u = 0; u < 2; ++u) {
                                     const int e = 4 * e4 + 2 * u;   // column within the chunk
-                                    const int x = 16 * c + e;       // query within the sub-tile
+                                    const int x = 16 * c + e;       // column among this thread's
                                     const uint64_t xs = f2_fma(f2_pack(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), c2x2,
                                                                f2_mul(lp[u], nl2e));
                                     float x0, x1;
@@ -938,18 +936,17 @@ __global__ void __launch_bounds__(BwdCfg<HD>::kThreads, 1) s2a_bwd_dkdv_kernel(c
                                 }
                             }
                         }
-                        tmem_st_32x8(tS + 16 * c, pkP);
-                        tmem_st_32x8(tS + 16 * c + 8, pkS);
+                        tmem_st_32x8(tS + 16 * cg, pkP);
+                        tmem_st_32x8(tS + 16 * cg + 8, pkS);
                         if constexpr (kSpill) {
                             // streaming stores: written once, read once by the dQ kernel much later
 #pragma unroll
                             for (int cc = 0; cc < 2; ++cc) {
                                 uint4 x = make_uint4(pkS[4 * cc], pkS[4 * cc + 1], pkS[4 * cc + 2], pkS[4 * cc + 3]);
                                 if (!key_valid) x = make_uint4(0u, 0u, 0u, 0u);
-                                __stcs(spill_dst + (2 * c + cc) * kTile, x);
+                                __stcs(spill_dst + (2 * cg + cc) * kTile, x);
                             }
                         }
-                        if (c < 3) tmem_wait_ld();
                     }
                     tmem_wait_st();
                     tc_fence_before();

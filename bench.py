@@ -39,10 +39,10 @@ FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_g
 NCU_TRAFFIC_8K = {
     "fwd": (249.6e6, 0.0),
     "bwd_preprocess": (137.9e6, 0.0),
-    "bwd_dkdv": None,                               # recomputing backward: persistent form not captured
+    "bwd_dkdv": (373.3e6, 0.0),                     # 270.7 MB read + 102.6 MB written
     "bwd_dq": (322.8e6, 0.0),
-    "bwd_dkdv_spill": (919.9e6 - 570.4e6, 570.4e6),  # 271.0 MB read + 648.9 MB written, 570.4 MB of it the spill
-    "bwd_dq_spill": (696.6e6 - 570.4e6, 570.4e6),    # 637.7 MB read + 58.9 MB written
+    "bwd_dkdv_spill": (920.2e6 - 570.4e6, 570.4e6),  # 270.9 MB read + 649.3 MB written, 570.4 MB of it the spill
+    "bwd_dq_spill": (695.9e6 - 570.4e6, 570.4e6),    # 637.6 MB read + 58.3 MB written
 }
 NCU_TRAFFIC_8K_SIZE = 1 * 8192 * (32 + 32) * 128
 NCU_SPILL_8K_BLOCKS = 32 * 4 * 16 * 17             # units x T (T + 1) blocks of 16 KiB, T = 2048 / 128

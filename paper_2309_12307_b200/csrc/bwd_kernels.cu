@@ -3,26 +3,29 @@
 // With P = exp(scale * Q K^T - lse) on the attended pairs and D_t = dO_t . o_t:
 //     dV = P^T dO          dP = dO V^T          dS = P o (dP - D)
 //     dQ = scale * dS K    dK = scale * dS^T Q
-// Three kernels:
+// Four kernels:
 //   1. preprocess: D[b,h,t] = sum_c dO[b,t,h,c] * o[b,t,h,c]                     (memory bound)
-//   2. dQ:   one CTA per 128-row query tile, walks the 128-key tiles of its group (keys <= query)
-//   3. dK,dV: one CTA per 128-row key tile, streams 64-query sub-tiles of every query head that
-//            shares the KV head (queries >= key), so the sum over those heads stays in tensor
-//            memory and needs no atomics.  It works on the transposed scores S^T = K Q^T so that
-//            P^T and dS^T come out with keys along tensor-memory lanes, which is the layout the
-//            A operand of dV += P^T dO and dK += dS^T Q needs.
+//   2. dQ, recomputing: one CTA per 128-row query tile, walks the 128-key tiles of its group (keys <=
+//            query) and computes S, dP, dS again
+//   3. dK,dV: persistent; a work item is one 128-row key tile, against which the 64-query sub-tiles of
+//            every query head that shares the KV head (queries >= key) are streamed, so the sum over
+//            those heads stays in tensor memory and needs no atomics.  It works on the transposed
+//            scores S^T = K Q^T so that P^T and dS^T come out with keys along tensor-memory lanes, which
+//            is the layout the A operand of dV += P^T dO and dK += dS^T Q needs.  Optionally it also
+//            leaves dS^T in global memory,
+//   4. dQ from spilled dS^T: persistent; a chain of plain products dQ_i = scale * sum_j dS_ij K_j that
+//            replaces kernel 2 when the caller's workspace has room for the spill.
 // The roll of the shifted heads and the group boundaries are folded into TMA coordinates exactly
 // as in the forward kernel; all results are stored at original token rows.
 //
-// Both tensor-core kernels use the same software pipeline (384 threads, one CTA per SM, all 512
-// tensor-memory columns): warp 0 loads with TMA; warp 1 issues the score MMAs and warp 2 the
-// gradient MMAs (a single issuing warp spends so long on its own barrier waits that the tensor pipe
-// runs dry in between; with two, one can issue while the other waits); warp 3 owns the tensor-memory
-// allocation; warps 4-11 do the elementwise work with one tensor-memory lane and half of the columns
-// per thread.  dP (dP^T) has a single buffer: the elementwise warps copy their part of it into
-// registers and release it at once, which leaves the columns for two (dQ: 128 wide) or three (dK,dV:
-// 64 wide) score buffers, so that the score products of later steps run while the elementwise warps
-// work on the current one.
+// Kernels 2 and 3 use the same warp roles (384 threads, one CTA per SM, all 512 tensor-memory columns):
+// warp 0 loads with TMA; warp 1 issues the score MMAs and warp 2 the gradient MMAs (a single issuing
+// warp spends so long on its own barrier waits that the tensor pipe runs dry in between; with two, one
+// can issue while the other waits); warp 3 owns the tensor-memory allocation; warps 4-11 do the
+// elementwise work with one tensor-memory lane and half of the columns per thread.  dP (dP^T) has a
+// single buffer: the elementwise warps copy their part of it into registers and release it at once,
+// which leaves the columns for two score buffers (and, in kernel 3, for K as a tensor-memory operand),
+// so that the score products of the next step run while the elementwise warps work on the current one.
 #include "s2a_params.h"
 #include "sm100_ptx.cuh"
 
@@ -114,23 +117,6 @@ __device__ __forceinline__ void store_acc_cols(uint32_t t_addr, float mul, __nv_
         }
     }
 }
-
-// Barrier block common to both kernels.
-template <int kStages>
-struct BwdBars {
-    uint64_t res_full;            // resident operands landed
-    uint64_t acc_full;            // all gradient MMAs done
-    uint64_t drain;               // abort path only (gradient MMA warp)
-    uint64_t drain2;              // abort path only (score MMA warp)
-    uint64_t s_full[3];           // S^T of a step is in tensor memory (buffer step % 3)
-    uint64_t p_full[3];           // bf16 P^T and dS^T of a step are in tensor memory
-    uint64_t buf_free[3];         // gradient MMAs that read a score buffer's bf16 operands are done
-    uint64_t dp_free;             // every elementwise thread holds its part of dP^T in registers
-    uint64_t st_full[kStages];    // streamed operands of a stage landed
-    uint64_t st_empty[kStages];   // MMAs reading a stage are done
-    uint32_t tmem_slot;
-    int abort_flag;
-};
 
 // ------------------------------------------------------------------------------------------------
 // 2. dQ

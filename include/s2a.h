@@ -90,7 +90,9 @@ int s2a_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
  *   in : q, k, v, o, lse (o and lse exactly as s2a_fwd produced them), dO
  *   out: dq, dk, dv (overwritten, not accumulated into)
  *   workspace: caller-owned device scratch of at least s2a_bwd_workspace_bytes(...) bytes,
- *              256-byte aligned; holds D[b,h,t] = dO[b,t,h,:] . o[b,t,h,:] in fp32.
+ *              256-byte aligned; holds D[b,h,t] = dO[b,t,h,:] . o[b,t,h,:] in fp32, the work counters of
+ *              the persistent kernels and, if it is large enough, the spilled dS (below).  Its contents
+ *              before the call do not matter; calls that can overlap on the GPU need a workspace each.
  * dk and dv sum over the H/Hkv query heads that share a KV head inside one thread block, and every dq
  * row is summed by one thread block in a fixed order, so the results are deterministic (no atomics).
  *
